@@ -1,0 +1,154 @@
+/*
+ * ac.h -- C ABI of the compressed-activation backward library (sm_100a).
+ *
+ * The method (paper: "Less Memory Means smaller GPUs: Backpropagation with
+ * Compressed Activations", Section 4 "Compressing Activation Maps" and its
+ * figure): a convolution layer computes its forward output from the full
+ * input X, but what it keeps for the backward pass is Z, the k x k average
+ * pooled copy of X, plus the pooling size and X's shape. In the backward pass
+ * the weight gradient is calculated as usual from Z inflated back to X's shape
+ * and the uncompressed output gradient dY. Input and bias gradients do not
+ * involve X and are not part of this library.
+ *
+ * Conventions common to every call
+ *   - All tensor pointers are DEVICE pointers unless a parameter says "host".
+ *     The caller owns every buffer (tensors and workspace). The library never
+ *     allocates or frees device memory and never synchronises, except where a
+ *     call says so; work is enqueued on `stream` (a cudaStream_t passed as
+ *     void*, NULL = the default stream).
+ *   - Tensor pointers must be 16-byte aligned (AC_ERR_MISALIGNED otherwise).
+ *   - Errors are return codes. No call aborts, throws or traps on the device.
+ *     The descriptor is validated before anything is launched.
+ *   - Reentrant; no global state except one-time kernel attribute set-up.
+ *
+ * Shapes (logical): X [N, C_in, H, W]; Z [N, C_in, ceil(H/k), ceil(W/k)];
+ * dY [N, C_out, H_o, W_o] with H_o = (H + 2 pad_h - R) / stride_h + 1 (floor),
+ * likewise W_o; dW [C_out, C_in, R, S]. Dilation 1, one group.
+ * Layout AC_NCHW stores X, Z, dY as [N][C][H][W] and dW as [C_out][C_in][R][S];
+ * AC_NHWC stores X, Z, dY as [N][H][W][C] and dW as [C_out][R][S][C_in].
+ * All buffers are dense (no strides).
+ */
+#ifndef AC_H_
+#define AC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    AC_OK = 0,
+    AC_ERR_INVALID_ARG = 1,         /* NULL pointer, non-positive size, bad enum, empty output */
+    AC_ERR_UNSUPPORTED = 2,         /* valid problem this build cannot run */
+    AC_ERR_MISALIGNED = 3,          /* a tensor or workspace pointer is not 16-byte aligned */
+    AC_ERR_WORKSPACE_TOO_SMALL = 4, /* workspace_bytes < ac_workspace_bytes(desc) */
+    AC_ERR_CUDA = 5,                /* a CUDA runtime call failed (launch, copy, attribute) */
+    AC_ERR_TIMEOUT = 6              /* a bounded wait inside a kernel ran out (see ac_workspace_status) */
+} ac_status;
+
+typedef enum { AC_F32 = 0, AC_BF16 = 1 } ac_dtype;
+typedef enum { AC_NCHW = 0, AC_NHWC = 1 } ac_layout;
+
+/* The problem statement of Section 4: the convolution layer, plus the pooling
+ * size k, which together with X's shape is all the metadata the stored Z needs. */
+typedef struct {
+    int32_t N, C_in, C_out, H, W;   /* X is N x C_in x H x W (logical) */
+    int32_t R, S;                   /* filter height, width */
+    int32_t stride_h, stride_w, pad_h, pad_w;
+    int32_t k;                      /* pooling factor, k >= 1; k = 1 stores X itself */
+    int32_t dtype;                  /* ac_dtype of X, Z, dY; dW is always fp32 */
+    int32_t layout;                 /* ac_layout of X, Z, dY and dW */
+} ac_conv_desc;
+
+/*
+ * Bytes of scratch that ac_conv2d_wgrad_compressed needs for this problem
+ * (split-K partial sums of dW plus a small status block). Pure host code.
+ * Returns 0 for an invalid descriptor.
+ */
+size_t ac_workspace_bytes(const ac_conv_desc *desc);
+
+/*
+ * Compression (Section 4; figure: mu_pq is the mean of the k x k block of X
+ * whose first element is X[pk, qk]). Z[n,c,p,q] = mean of X[n,c,h,w] over
+ * h in [pk, min(pk+k,H)), w in [qk, min(qk+k,W)): blocks are aligned to X's
+ * index 0; a partial last block is averaged over the elements it has. The sum
+ * is formed in fp32 and rounded once to the storage dtype.
+ *
+ *   x      in : [N,C_in,H,W] in desc->layout / desc->dtype. With y_out == NULL
+ *               this is the activation X itself.
+ *   z      out: [N,C_in,ceil(H/k),ceil(W/k)], same layout and dtype.
+ *   y_out  out, optional: if non-NULL the call is the fused form for a layer
+ *               whose input is produced by a ReLU: x is the pre-activation A,
+ *               y_out = max(A, 0) (same shape as x; may be the same pointer as
+ *               x for in-place ReLU) and z = pooling of y_out.
+ * Only N, C_in, H, W, k, dtype and layout of the descriptor are used.
+ * One kernel launch on `stream`; no scratch memory.
+ */
+ac_status ac_compress(const ac_conv_desc *desc, const void *x, void *z,
+                      void *y_out, void *stream);
+
+/*
+ * Weight gradient from the compressed activation (Section 4: inflate Z to the
+ * original dimensions, then calculate the weight gradient normally; figure:
+ * dL/dW ~ Z (*) dL/dY). With Xt[n,c,h,w] = Z[n,c,h/k,w/k] for 0<=h<H, 0<=w<W
+ * and 0 elsewhere (the convolution's zero padding, applied after inflation):
+ *
+ *   dW[co,ci,r,s] = sum_{n,ho,wo} dY[n,co,ho,wo] * Xt[n,ci,ho*stride_h-pad_h+r,
+ *                                                          wo*stride_w-pad_w+s]
+ *
+ * Xt is never written to memory. Products are accumulated in fp32.
+ *
+ *   z          in : as produced by ac_compress.
+ *   dy         in : [N,C_out,H_o,W_o], desc->layout / desc->dtype.
+ *   dw         out: fp32, OVERWRITTEN (not accumulated into); layout per desc->layout.
+ *   workspace     : device scratch of at least ac_workspace_bytes(desc) bytes,
+ *                   16-byte aligned; contents on entry are ignored, contents on
+ *                   exit are unspecified except for the status block read by
+ *                   ac_workspace_status. Two calls that overlap on the device
+ *                   must not share a workspace.
+ * Returns AC_ERR_WORKSPACE_TOO_SMALL / AC_ERR_MISALIGNED / AC_ERR_INVALID_ARG
+ * before launching anything. Results are deterministic (fixed summation order).
+ */
+ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc *desc, const void *z,
+                                     const void *dy, float *dw, void *workspace,
+                                     size_t workspace_bytes, void *stream);
+
+/*
+ * Reads back the status block a previous ac_conv2d_wgrad_compressed call left
+ * in `workspace`: synchronises `stream`, then returns AC_OK, or AC_ERR_TIMEOUT
+ * if a bounded wait inside a kernel gave up (dW is then not valid), or
+ * AC_ERR_CUDA if the stream reports an error. `detail`, if non-NULL, receives
+ * a kernel-specific code saying which wait ran out (0 when AC_OK).
+ */
+ac_status ac_workspace_status(const void *workspace, void *stream, uint32_t *detail);
+
+/*
+ * One backward step of a compressed layer on HOST buffers (Section 4, whole
+ * path): copies X and dY to the device, compresses X to Z, computes dW from Z
+ * and dY, copies dW back. For callers that hold their tensors in host memory
+ * and for end-to-end timing.
+ *
+ *   x_host, dy_host in : host memory (pinned for asynchronous copies),
+ *                        desc->layout / desc->dtype.
+ *   dw_host        out : host memory, fp32.
+ *   z_host    optional : if non-NULL also receives Z (desc->dtype).
+ *   arena              : DEVICE scratch of at least ac_host_step_arena_bytes(desc)
+ *                        bytes, 256-byte aligned; holds X, Z, dY, dW and the
+ *                        wgrad workspace for the duration of the call.
+ * Enqueues the copies and kernels on `stream` and returns without waiting;
+ * the caller synchronises the stream before reading dw_host.
+ */
+size_t ac_host_step_arena_bytes(const ac_conv_desc *desc);
+ac_status ac_backward_step_host(const ac_conv_desc *desc, const void *x_host,
+                                const void *dy_host, float *dw_host, void *z_host,
+                                void *arena, size_t arena_bytes, void *stream);
+
+/* Static, human-readable name of a status code. */
+const char *ac_status_string(ac_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AC_H_ */

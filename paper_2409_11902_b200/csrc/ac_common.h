@@ -1,0 +1,70 @@
+// Internal definitions shared by the translation units of libac (not installed).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ac.h"
+
+namespace ac {
+
+constexpr int kNumSMs = 148;               // B200: the only target of this library
+constexpr size_t kStatusBlockBytes = 256;  // first bytes of every wgrad workspace
+
+// Derived sizes of a validated descriptor.
+struct Dims {
+    int N, Ci, Co, H, W, R, S, sh, sw, ph, pw, k;
+    int Hp, Wp;   // pooled size (ceil)
+    int Ho, Wo;   // convolution output size
+    int dtype, layout;
+    int elt;      // bytes per element of X, Z, dY
+    long long x_elems() const { return (long long)N * Ci * H * W; }
+    long long z_elems() const { return (long long)N * Ci * Hp * Wp; }
+    long long dy_elems() const { return (long long)N * Co * Ho * Wo; }
+    long long dw_elems() const { return (long long)Co * Ci * R * S; }
+    long long K() const { return (long long)N * Ho * Wo; }
+};
+
+// Validates and expands a descriptor. `need_conv` = false checks only the
+// fields ac_compress uses.
+ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* out);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- wgrad planning (pure host arithmetic; decides kernel and split-K) ------
+enum WgradPath { PATH_SIMT = 0, PATH_TC = 1 };
+
+struct WgradPlan {
+    int path;        // WgradPath
+    int splits;      // K-slices whose partial dW tensors are summed in fixed order
+    // SIMT path: each slice covers `simt_k_per_split` flattened (n,ho,wo) positions
+    long long simt_k_per_split;
+    // tensor-core path
+    int tc_band;     // output rows per K-tile
+    int tc_groups;   // CTAs sharing one K-slice, each owning part of the output
+    int tc_ktiles;   // K-tiles in the whole problem
+    int tc_stages;   // shared-memory pipeline depth
+    size_t bytes;    // workspace bytes including the status block
+};
+
+WgradPlan plan_wgrad(const Dims& d);
+
+// ---- launchers (each enqueues on `stream`, returns AC_OK or AC_ERR_CUDA) -----
+ac_status launch_compress(const Dims& d, const void* x, void* z, void* y_out, cudaStream_t stream);
+ac_status launch_wgrad_simt(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
+                            float* dw, void* workspace, cudaStream_t stream);
+bool tc_supported(const Dims& d);
+void plan_tc(const Dims& d, WgradPlan* p);
+ac_status launch_wgrad_tc(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
+                          float* dw, void* workspace, cudaStream_t stream);
+ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
+                               cudaStream_t stream);
+
+#define AC_CUDA_TRY(expr)                           \
+    do {                                            \
+        cudaError_t e__ = (expr);                   \
+        if (e__ != cudaSuccess) return AC_ERR_CUDA; \
+    } while (0)
+
+}  // namespace ac
