@@ -1,0 +1,10 @@
+"""Backpropagation with pooling-compressed activations: B200 (sm_100a) hot path.
+
+`api` binds the C-ABI CUDA library (libac.so, built in-tree from csrc/);
+`synth` draws the seeded synthetic inputs used by the tests and the benchmark.
+"""
+from . import synth  # noqa: F401
+from .api import (  # noqa: F401
+    AcError, ConvDesc, ac_backward_step_host, ac_compress, ac_conv2d_wgrad_compressed,
+    ac_host_step_arena_bytes, ac_workspace_bytes, ac_workspace_status, status_string,
+)

@@ -1,0 +1,167 @@
+// C-ABI entry points: argument validation, planning, dispatch. See include/ac.h.
+#include "ac_common.h"
+
+namespace ac {
+
+ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o) {
+    if (!d || !o) return AC_ERR_INVALID_ARG;
+    if (d->N <= 0 || d->C_in <= 0 || d->H <= 0 || d->W <= 0 || d->k <= 0) return AC_ERR_INVALID_ARG;
+    if (d->dtype != AC_F32 && d->dtype != AC_BF16) return AC_ERR_INVALID_ARG;
+    if (d->layout != AC_NCHW && d->layout != AC_NHWC) return AC_ERR_INVALID_ARG;
+    o->N = d->N; o->Ci = d->C_in; o->H = d->H; o->W = d->W; o->k = d->k;
+    o->dtype = d->dtype; o->layout = d->layout;
+    o->elt = d->dtype == AC_F32 ? 4 : 2;
+    o->Hp = (d->H + d->k - 1) / d->k;
+    o->Wp = (d->W + d->k - 1) / d->k;
+    o->Co = 1; o->R = 1; o->S = 1; o->sh = 1; o->sw = 1; o->ph = 0; o->pw = 0;
+    o->Ho = d->H; o->Wo = d->W;
+    const long long lim = 1ll << 40;  // elements; far above 180 GB of any dtype
+    if ((long long)d->N * d->C_in * d->H * d->W >= lim) return AC_ERR_INVALID_ARG;
+    if (!need_conv) return AC_OK;
+    if (d->C_out <= 0 || d->R <= 0 || d->S <= 0 || d->stride_h <= 0 || d->stride_w <= 0 ||
+        d->pad_h < 0 || d->pad_w < 0)
+        return AC_ERR_INVALID_ARG;
+    if (d->H + 2 * (long long)d->pad_h < d->R || d->W + 2 * (long long)d->pad_w < d->S)
+        return AC_ERR_INVALID_ARG;  // empty output
+    o->Co = d->C_out; o->R = d->R; o->S = d->S;
+    o->sh = d->stride_h; o->sw = d->stride_w; o->ph = d->pad_h; o->pw = d->pad_w;
+    o->Ho = (d->H + 2 * d->pad_h - d->R) / d->stride_h + 1;
+    o->Wo = (d->W + 2 * d->pad_w - d->S) / d->stride_w + 1;
+    if ((long long)d->N * d->C_out * o->Ho * o->Wo >= lim) return AC_ERR_INVALID_ARG;
+    if ((long long)d->C_out * d->C_in * d->R * d->S >= (1ll << 31)) return AC_ERR_INVALID_ARG;
+    if ((long long)d->C_in * d->R * d->S >= (1ll << 31)) return AC_ERR_INVALID_ARG;
+    return AC_OK;
+}
+
+static inline long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
+
+WgradPlan plan_wgrad(const Dims& d) {
+    WgradPlan p{};
+    if (tc_supported(d)) {
+        p.path = PATH_TC;
+        plan_tc(d, &p);
+        return p;
+    }
+    p.path = PATH_SIMT;
+    const long long K = d.K();
+    const long long J = (long long)d.Ci * d.R * d.S;
+    const long long tiles = ceil_div(d.Co, 64) * ceil_div(J, 64);
+    // enough blocks to fill the chip four times over, slices of 256..2048
+    // positions so that each fp32 running sum stays short
+    long long want = ceil_div(4 * kNumSMs, tiles);
+    long long kps = ceil_div(ceil_div(K, want), 16) * 16;
+    if (kps < 256) kps = 256;
+    if (kps > 2048) kps = 2048;
+    const long long dw_bytes = d.dw_elems() * 4;
+    long long max_splits = (256ll << 20) / dw_bytes;
+    if (max_splits < 1) max_splits = 1;
+    if (max_splits > 65535) max_splits = 65535;
+    if (ceil_div(K, kps) > max_splits) kps = ceil_div(ceil_div(K, max_splits), 16) * 16;
+    p.simt_k_per_split = kps;
+    p.splits = (int)ceil_div(K, kps);
+    p.bytes = kStatusBlockBytes + (p.splits > 1 ? (size_t)p.splits * dw_bytes : 0);
+    return p;
+}
+
+}  // namespace ac
+
+using namespace ac;
+
+extern "C" {
+
+size_t ac_workspace_bytes(const ac_conv_desc* desc) {
+    Dims d;
+    if (make_dims(desc, true, &d) != AC_OK) return 0;
+    return plan_wgrad(d).bytes;
+}
+
+ac_status ac_compress(const ac_conv_desc* desc, const void* x, void* z, void* y_out, void* stream) {
+    Dims d;
+    ac_status st = make_dims(desc, false, &d);
+    if (st != AC_OK) return st;
+    if (!x || !z) return AC_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(z) || !aligned16(y_out)) return AC_ERR_MISALIGNED;
+    return launch_compress(d, x, z, y_out, static_cast<cudaStream_t>(stream));
+}
+
+ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, const void* dy,
+                                     float* dw, void* workspace, size_t workspace_bytes,
+                                     void* stream) {
+    Dims d;
+    ac_status st = make_dims(desc, true, &d);
+    if (st != AC_OK) return st;
+    if (!z || !dy || !dw || !workspace) return AC_ERR_INVALID_ARG;
+    if (!aligned16(z) || !aligned16(dy) || !aligned16(dw) || !aligned16(workspace))
+        return AC_ERR_MISALIGNED;
+    const WgradPlan p = plan_wgrad(d);
+    if (workspace_bytes < p.bytes) return AC_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
+    if (p.path == PATH_TC) return launch_wgrad_tc(d, p, z, dy, dw, workspace, s);
+    return launch_wgrad_simt(d, p, z, dy, dw, workspace, s);
+}
+
+ac_status ac_workspace_status(const void* workspace, void* stream, uint32_t* detail) {
+    if (!workspace) return AC_ERR_INVALID_ARG;
+    uint32_t word[2] = {0, 0};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    AC_CUDA_TRY(cudaMemcpyAsync(word, workspace, sizeof(word), cudaMemcpyDeviceToHost, s));
+    AC_CUDA_TRY(cudaStreamSynchronize(s));
+    if (detail) *detail = word[1];
+    return word[0] == 0 ? AC_OK : AC_ERR_TIMEOUT;
+}
+
+static inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+size_t ac_host_step_arena_bytes(const ac_conv_desc* desc) {
+    Dims d;
+    if (make_dims(desc, true, &d) != AC_OK) return 0;
+    return up256((size_t)d.x_elems() * d.elt) + up256((size_t)d.z_elems() * d.elt) +
+           up256((size_t)d.dy_elems() * d.elt) + up256((size_t)d.dw_elems() * 4) +
+           up256(plan_wgrad(d).bytes);
+}
+
+ac_status ac_backward_step_host(const ac_conv_desc* desc, const void* x_host, const void* dy_host,
+                                float* dw_host, void* z_host, void* arena, size_t arena_bytes,
+                                void* stream) {
+    Dims d;
+    ac_status st = make_dims(desc, true, &d);
+    if (st != AC_OK) return st;
+    if (!x_host || !dy_host || !dw_host || !arena) return AC_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(arena) & 255u) return AC_ERR_MISALIGNED;
+    if (arena_bytes < ac_host_step_arena_bytes(desc)) return AC_ERR_WORKSPACE_TOO_SMALL;
+    const size_t xb = (size_t)d.x_elems() * d.elt, zb = (size_t)d.z_elems() * d.elt;
+    const size_t gb = (size_t)d.dy_elems() * d.elt, wb = (size_t)d.dw_elems() * 4;
+    char* base = static_cast<char*>(arena);
+    void* x = base;
+    void* z = base + up256(xb);
+    void* dy = base + up256(xb) + up256(zb);
+    float* dw = reinterpret_cast<float*>(base + up256(xb) + up256(zb) + up256(gb));
+    void* ws = base + up256(xb) + up256(zb) + up256(gb) + up256(wb);
+    const size_t ws_bytes = plan_wgrad(d).bytes;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    AC_CUDA_TRY(cudaMemcpyAsync(x, x_host, xb, cudaMemcpyHostToDevice, s));
+    AC_CUDA_TRY(cudaMemcpyAsync(dy, dy_host, gb, cudaMemcpyHostToDevice, s));
+    st = ac_compress(desc, x, z, nullptr, stream);
+    if (st != AC_OK) return st;
+    st = ac_conv2d_wgrad_compressed(desc, z, dy, dw, ws, ws_bytes, stream);
+    if (st != AC_OK) return st;
+    AC_CUDA_TRY(cudaMemcpyAsync(dw_host, dw, wb, cudaMemcpyDeviceToHost, s));
+    if (z_host) AC_CUDA_TRY(cudaMemcpyAsync(z_host, z, zb, cudaMemcpyDeviceToHost, s));
+    return AC_OK;
+}
+
+const char* ac_status_string(ac_status status) {
+    switch (status) {
+        case AC_OK: return "AC_OK";
+        case AC_ERR_INVALID_ARG: return "AC_ERR_INVALID_ARG";
+        case AC_ERR_UNSUPPORTED: return "AC_ERR_UNSUPPORTED";
+        case AC_ERR_MISALIGNED: return "AC_ERR_MISALIGNED";
+        case AC_ERR_WORKSPACE_TOO_SMALL: return "AC_ERR_WORKSPACE_TOO_SMALL";
+        case AC_ERR_CUDA: return "AC_ERR_CUDA";
+        case AC_ERR_TIMEOUT: return "AC_ERR_TIMEOUT";
+    }
+    return "AC_ERR_UNKNOWN";
+}
+
+}  // extern "C"

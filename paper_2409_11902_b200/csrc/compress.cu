@@ -1,0 +1,277 @@
+// Compression kernels: Z = k x k average pooling of the convolution input X
+// (Section 4 of the paper; blocks aligned to X's index 0, partial edge blocks
+// averaged over the elements they have), optionally fused with the ReLU that
+// produces X. Bandwidth bound: every element of X is read once with 16-byte
+// loads, sums are formed in fp32 registers (plus one warp shuffle where a
+// block spans two lanes), Z is written once.
+#include "ac_common.h"
+
+namespace ac {
+namespace {
+
+template <typename T> struct VecTraits;
+template <> struct VecTraits<float> { static constexpr int VW = 4; };
+template <> struct VecTraits<__nv_bfloat16> { static constexpr int VW = 8; };
+
+// 16-byte global load; streaming hint when the buffer is only read.
+template <bool STREAM>
+__device__ __forceinline__ uint4 load16(const void* p) {
+    if (STREAM) return __ldcs(reinterpret_cast<const uint4*>(p));
+    return *reinterpret_cast<const uint4*>(p);
+}
+
+template <typename T, bool RELU>
+__device__ __forceinline__ void unpack(uint4& raw, float* f);
+
+template <>
+__device__ __forceinline__ void unpack<float, false>(uint4& raw, float* f) {
+    f[0] = __uint_as_float(raw.x); f[1] = __uint_as_float(raw.y);
+    f[2] = __uint_as_float(raw.z); f[3] = __uint_as_float(raw.w);
+}
+template <>
+__device__ __forceinline__ void unpack<float, true>(uint4& raw, float* f) {
+    f[0] = fmaxf(__uint_as_float(raw.x), 0.f); f[1] = fmaxf(__uint_as_float(raw.y), 0.f);
+    f[2] = fmaxf(__uint_as_float(raw.z), 0.f); f[3] = fmaxf(__uint_as_float(raw.w), 0.f);
+    raw = make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                     __float_as_uint(f[3]));
+}
+__device__ __forceinline__ void bf2_to_f(uint32_t u, float& lo, float& hi) {
+    lo = __uint_as_float(u << 16);
+    hi = __uint_as_float(u & 0xffff0000u);
+}
+// max(x,0) on two packed bf16: clear each half whose sign bit is set
+// (-0 and negative NaN payloads also become +0, like fmaxf(x, 0)).
+__device__ __forceinline__ uint32_t relu_bf2(uint32_t u) {
+    uint32_t m = 0;
+    if (!(u & 0x00008000u)) m |= 0x0000ffffu;
+    if (!(u & 0x80000000u)) m |= 0xffff0000u;
+    return u & m;
+}
+template <>
+__device__ __forceinline__ void unpack<__nv_bfloat16, false>(uint4& raw, float* f) {
+    bf2_to_f(raw.x, f[0], f[1]); bf2_to_f(raw.y, f[2], f[3]);
+    bf2_to_f(raw.z, f[4], f[5]); bf2_to_f(raw.w, f[6], f[7]);
+}
+template <>
+__device__ __forceinline__ void unpack<__nv_bfloat16, true>(uint4& raw, float* f) {
+    raw.x = relu_bf2(raw.x); raw.y = relu_bf2(raw.y);
+    raw.z = relu_bf2(raw.z); raw.w = relu_bf2(raw.w);
+    unpack<__nv_bfloat16, false>(raw, f);
+}
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) {
+    return __float2bfloat16_rn(v);
+}
+
+template <typename T>
+__device__ __forceinline__ uint4 pack(const float* f);
+template <>
+__device__ __forceinline__ uint4 pack<float>(const float* f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                      __float_as_uint(f[3]));
+}
+__device__ __forceinline__ uint32_t f2_to_bf2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+template <>
+__device__ __forceinline__ uint4 pack<__nv_bfloat16>(const float* f) {
+    return make_uint4(f2_to_bf2(f[0], f[1]), f2_to_bf2(f[2], f[3]), f2_to_bf2(f[4], f[5]),
+                      f2_to_bf2(f[6], f[7]));
+}
+
+// ---- NHWC, C a multiple of the vector width --------------------------------
+// One thread per output vector (n, p, q, 16 bytes of channels): k*k independent
+// 16-byte loads, element-wise fp32 sums, one 16-byte store. Adjacent threads
+// hold adjacent channel vectors, so every warp-wide access is contiguous.
+template <typename T, bool RELU>
+__global__ void __launch_bounds__(256)
+compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W, int CV, int k,
+                  int Hp, int Wp, long long total) {
+    constexpr int VW = VecTraits<T>::VW;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int cv = (int)(idx % CV);
+    long long t = idx / CV;
+    const int q = (int)(t % Wp); t /= Wp;
+    const int p = (int)(t % Hp);
+    const long long n = t / Hp;
+    const int h0 = p * k, w0 = q * k;
+    const int h1 = min(h0 + k, H), w1 = min(w0 + k, W);
+    float acc[VW];
+#pragma unroll
+    for (int i = 0; i < VW; ++i) acc[i] = 0.f;
+    for (int h = h0; h < h1; ++h) {
+        float row[VW];
+#pragma unroll
+        for (int i = 0; i < VW; ++i) row[i] = 0.f;
+        const long long rbase = ((n * H + h) * (long long)W) * CV + cv;
+        for (int w = w0; w < w1; ++w) {
+            const long long off = (rbase + (long long)w * CV) * VW;
+            uint4 raw = load16<!RELU>(x + off);
+            float f[VW];
+            unpack<T, RELU>(raw, f);
+            if (RELU) *reinterpret_cast<uint4*>(y + off) = raw;
+#pragma unroll
+            for (int i = 0; i < VW; ++i) row[i] += f[i];
+        }
+#pragma unroll
+        for (int i = 0; i < VW; ++i) acc[i] += row[i];
+    }
+    const float inv = 1.0f / (float)((h1 - h0) * (w1 - w0));
+#pragma unroll
+    for (int i = 0; i < VW; ++i) acc[i] *= inv;
+    *reinterpret_cast<uint4*>(z + idx * VW) = pack<T>(acc);
+}
+
+// ---- NCHW, W a multiple of the vector width and of k, k in {2,4,8} ---------
+// One thread per (plane, pooled row, 16-byte column chunk): lanes of a warp
+// read consecutive 16-byte chunks of a row. Vertical sums over the k rows are
+// element-wise; the horizontal sum is a tree inside the vector, finished with
+// one warp shuffle when a block spans two lanes (fp32, k = 8).
+template <typename T, int K, bool RELU>
+__global__ void __launch_bounds__(256)
+compress_nchw_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W, int Hp, int Wp,
+                  long long total) {
+    constexpr int VW = VecTraits<T>::VW;
+    const int WV = W / VW;
+    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool active = idx < total;
+    if (!active) idx = total - 1;  // keep whole warps alive for the shuffle
+    const int wv = (int)(idx % WV);
+    long long t = idx / WV;
+    const int p = (int)(t % Hp);
+    const long long nc = t / Hp;
+    const int h0 = p * K;
+    const int h1 = min(h0 + K, H);
+    float acc[VW];
+#pragma unroll
+    for (int i = 0; i < VW; ++i) acc[i] = 0.f;
+#pragma unroll
+    for (int dh = 0; dh < K; ++dh) {
+        const int h = h0 + dh;
+        if (h < h1) {
+            const long long off = ((nc * H + h) * (long long)WV + wv) * VW;
+            uint4 raw = load16<!RELU>(x + off);
+            float f[VW];
+            unpack<T, RELU>(raw, f);
+            if (RELU && active) *reinterpret_cast<uint4*>(y + off) = raw;
+#pragma unroll
+            for (int i = 0; i < VW; ++i) acc[i] += f[i];
+        }
+    }
+    const float inv = 1.0f / (float)((h1 - h0) * K);
+    if (K <= VW) {
+        constexpr int NO = (K <= VW) ? VW / K : 1;  // outputs per thread
+        float out[NO];
+#pragma unroll
+        for (int j = 0; j < NO; ++j) {
+            // pairwise tree over the K partial sums of output j
+            float s[K];
+#pragma unroll
+            for (int i = 0; i < K; ++i) s[i] = acc[(j * K + i) % VW];
+#pragma unroll
+            for (int w = K / 2; w >= 1; w /= 2)
+#pragma unroll
+                for (int i = 0; i < w; ++i) s[i] += s[i + w];
+            out[j] = s[0] * inv;
+        }
+        if (active) {
+            T* zp = z + (nc * Hp + p) * (long long)Wp + (long long)wv * NO;
+#pragma unroll
+            for (int j = 0; j < NO; ++j) zp[j] = from_f<T>(out[j]);
+        }
+    } else {
+        // K == 2 * VW: lanes 2j and 2j+1 hold the two halves of one block
+        float s = (acc[0] + acc[1 % VW]) + (acc[2 % VW] + acc[3 % VW]);
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        if (active && (wv & 1) == 0)
+            z[(nc * Hp + p) * (long long)Wp + (wv >> 1)] = from_f<T>(s * inv);
+    }
+}
+
+// ---- any layout, any k, any size: one thread per element of Z ---------------
+template <typename T, bool RELU>
+__global__ void __launch_bounds__(256)
+compress_generic(const T* x, T* __restrict__ z, T* y, int C, int H, int W, int k, int Hp, int Wp,
+                 int nhwc, long long total) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    int c, p, q;
+    long long n, t = idx;
+    if (nhwc) { c = (int)(t % C); t /= C; q = (int)(t % Wp); t /= Wp; p = (int)(t % Hp); n = t / Hp; }
+    else      { q = (int)(t % Wp); t /= Wp; p = (int)(t % Hp); t /= Hp; c = (int)(t % C); n = t / C; }
+    const int h0 = p * k, w0 = q * k;
+    const int h1 = min(h0 + k, H), w1 = min(w0 + k, W);
+    float acc = 0.f;
+    for (int h = h0; h < h1; ++h) {
+        float row = 0.f;
+        for (int w = w0; w < w1; ++w) {
+            const long long off = nhwc ? ((n * H + h) * (long long)W + w) * C + c
+                                       : ((n * C + c) * (long long)H + h) * W + w;
+            float v = to_f(x[off]);
+            if (RELU) { v = fmaxf(v, 0.f); y[off] = from_f<T>(v); }
+            row += v;
+        }
+        acc += row;
+    }
+    z[idx] = from_f<T>(acc * (1.0f / (float)((h1 - h0) * (w1 - w0))));
+}
+
+inline unsigned blocks_for(long long total) { return (unsigned)((total + 255) / 256); }
+
+template <typename T, bool RELU>
+ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, cudaStream_t st) {
+    constexpr int VW = VecTraits<T>::VW;
+    const long long zt = d.z_elems();
+    if (zt >= (1ll << 31) * 256) return AC_ERR_UNSUPPORTED;
+    const bool pow2k = d.k == 2 || d.k == 4 || d.k == 8;
+    if (d.k == 1 && d.x_elems() % VW == 0) {
+        // a copy (or a plain ReLU): treat the tensor as one row of 16-byte vectors
+        const long long nv = d.x_elems() / VW;
+        if (nv < (1ll << 31)) {
+            compress_nhwc_vec<T, RELU><<<blocks_for(nv), 256, 0, st>>>(x, z, y, 1, (int)nv, 1, 1, 1,
+                                                                       (int)nv, nv);
+            AC_CUDA_TRY(cudaGetLastError());
+            return AC_OK;
+        }
+    }
+    if (d.layout == AC_NHWC && d.Ci % VW == 0) {
+        const long long total = zt / VW;
+        compress_nhwc_vec<T, RELU><<<blocks_for(total), 256, 0, st>>>(x, z, y, d.H, d.W, d.Ci / VW,
+                                                                      d.k, d.Hp, d.Wp, total);
+    } else if (d.layout == AC_NCHW && pow2k && d.W % VW == 0 && d.W % d.k == 0 &&
+               (VW % d.k == 0 || d.k == 2 * VW)) {
+        const long long total = (long long)d.N * d.Ci * d.Hp * (d.W / VW);
+        const unsigned g = blocks_for(total);
+        if (d.k == 2)
+            compress_nchw_vec<T, 2, RELU><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp, total);
+        else if (d.k == 4)
+            compress_nchw_vec<T, 4, RELU><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp, total);
+        else
+            compress_nchw_vec<T, 8, RELU><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp, total);
+    } else {
+        compress_generic<T, RELU><<<blocks_for(zt), 256, 0, st>>>(
+            x, z, y, d.Ci, d.H, d.W, d.k, d.Hp, d.Wp, d.layout == AC_NHWC, zt);
+    }
+    AC_CUDA_TRY(cudaGetLastError());
+    return AC_OK;
+}
+
+}  // namespace
+
+ac_status launch_compress(const Dims& d, const void* x, void* z, void* y_out, cudaStream_t st) {
+    if (d.dtype == AC_F32) {
+        return y_out ? launch_typed<float, true>(d, (const float*)x, (float*)z, (float*)y_out, st)
+                     : launch_typed<float, false>(d, (const float*)x, (float*)z, nullptr, st);
+    }
+    using B = __nv_bfloat16;
+    return y_out ? launch_typed<B, true>(d, (const B*)x, (B*)z, (B*)y_out, st)
+                 : launch_typed<B, false>(d, (const B*)x, (B*)z, nullptr, st);
+}
+
+}  // namespace ac
