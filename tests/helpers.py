@@ -1,0 +1,139 @@
+"""Shared machinery of the GPU parity tests: run the CUDA library through its
+C ABI on seeded inputs and compare with the CPU checker (oracle/)."""
+import numpy as np
+import torch
+
+import oracle
+import paper_2409_11902_b200 as ac
+from paper_2409_11902_b200 import synth
+
+CANARY = 0x5A
+
+# Tolerances (stated by the benchmark spec for this path):
+#   fp32 compress: max relative error <= 1e-6 (relative to the block's mean |x|)
+#   bf16 compress: one rounding to bf16 (half an ulp = 2^-9 .. 2^-8 relative) on top
+#   dW: relative Frobenius error <= 1e-5 (fp32 inputs), <= 1e-2 (bf16 inputs, fp32 accumulate)
+TOL_Z = {"f32": 1e-6, "bf16": 2.0 ** -8 * 1.001 + 1e-6}
+TOL_DW = {"f32": 1e-5, "bf16": 1e-2}
+
+
+def padded_empty(shape, dtype, dev, pad_bytes=512):
+    """A device tensor of `shape` carved from a larger byte buffer filled with a
+    canary, so that writes outside the tensor can be detected afterwards."""
+    n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+    n_al = (n + 255) // 256 * 256
+    buf = torch.full((pad_bytes + n_al + pad_bytes,), CANARY, dtype=torch.uint8, device=dev)
+    view = buf[pad_bytes:pad_bytes + n].view(dtype).view(shape)
+    return buf, view, (pad_bytes, n)
+
+
+def canary_intact(buf, span):
+    lo, n = span
+    b = buf.cpu()
+    return bool((b[:lo] == CANARY).all()) and bool((b[lo + n:] == CANARY).all())
+
+
+def compress_error(z_got_nchw: np.ndarray, x_nchw: np.ndarray, k: int):
+    """max_i |z_i - zhat_i| / mean_{block i} |x|; blocks whose inputs are all
+    zero must give exactly 0."""
+    z_ref = oracle.pool(x_nchw, k)
+    denom = oracle.pool(np.abs(x_nchw), k)
+    diff = np.abs(z_got_nchw - z_ref)
+    zero = denom == 0
+    assert not diff[zero].any(), "all-zero block must pool to exactly 0"
+    return float(np.max(diff[~zero] / denom[~zero])) if (~zero).any() else 0.0
+
+
+def run_compress(d: ac.ConvDesc, seed=0, fused_relu=False, inplace=False, dev="cuda:0"):
+    """Returns (error, z as NCHW float64, x as NCHW float64 (post-ReLU))."""
+    shape = (d.N, d.C_in, d.H, d.W)
+    if fused_relu:
+        a = synth.pre_activation(seed, shape, d.dtype)
+        x64 = oracle.relu(synth.to_f64(a))
+        src = a
+    else:
+        src = synth.activation(seed, shape, d.dtype)
+        x64 = synth.to_f64(src)
+    xd = synth.to_layout(src, d.layout).to(dev)
+    zbuf, z, zspan = padded_empty(d.z_shape, d.torch_dtype, dev)
+    ybuf = y = None
+    if fused_relu:
+        if inplace:
+            y = xd
+        else:
+            ybuf, y, yspan = padded_empty(d.x_shape, d.torch_dtype, dev)
+    ac.ac_compress(d, xd, z, y)
+    torch.cuda.synchronize()
+    assert canary_intact(zbuf, zspan), "ac_compress wrote outside Z"
+    if ybuf is not None:
+        assert canary_intact(ybuf, yspan), "ac_compress wrote outside Y"
+    if fused_relu:
+        y64 = synth.to_f64(synth.from_layout(y.cpu(), d.layout))
+        assert np.array_equal(y64, x64), "fused ReLU output differs from max(A, 0)"
+    z64 = synth.to_f64(synth.from_layout(z.cpu(), d.layout))
+    return compress_error(z64, x64, d.k), z64, x64
+
+
+def make_wgrad_inputs(d: ac.ConvDesc, seed=0):
+    """X -> Z by the checker's pooling, rounded once to the storage dtype, so
+    that the checker and the GPU read identical bits of Z and dY."""
+    x = synth.activation(seed, (d.N, d.C_in, d.H, d.W), d.dtype)
+    z = synth.to_storage(oracle.pool(synth.to_f64(x), d.k), d.dtype)
+    dy = synth.grad_output(seed, (d.N, d.C_out, d.Ho, d.Wo), d.dtype)
+    return z, dy
+
+
+def dw_to_oihw(dw: torch.Tensor, layout: str) -> np.ndarray:
+    a = dw.detach().cpu().double().numpy()
+    return a.transpose(0, 3, 1, 2) if layout == "nhwc" else a
+
+
+def run_wgrad(d: ac.ConvDesc, z, dy, dev="cuda:0", repeat=2):
+    """Runs the library `repeat` times (bitwise-equal results required) and
+    returns dW as float64 [Co,Ci,R,S]."""
+    zd = synth.to_layout(z, d.layout).to(dev)
+    dyd = synth.to_layout(dy, d.layout).to(dev)
+    nbytes = ac.ac_workspace_bytes(d)
+    assert nbytes > 0
+    outs = []
+    for it in range(repeat):
+        wbuf, dw, wspan = padded_empty(d.dw_shape, torch.float32, dev)
+        sbuf, ws, sspan = padded_empty((nbytes,), torch.uint8, dev)
+        if it == 1:
+            ws.fill_(0xFF)          # workspace contents on entry must not matter
+            dw.fill_(float("nan"))  # dW is overwritten, not accumulated into
+        ac.ac_conv2d_wgrad_compressed(d, zd, dyd, dw, ws, nbytes)
+        st, detail = ac.ac_workspace_status(ws)
+        assert st == 0, f"device status {st} detail {detail:#x}"
+        assert canary_intact(wbuf, wspan), "wgrad wrote outside dW"
+        assert canary_intact(sbuf, sspan), "wgrad wrote outside the workspace"
+        outs.append(dw.clone())
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0]), "results differ between identical calls"
+    return dw_to_oihw(outs[0], d.layout)
+
+
+def wgrad_error_full(d: ac.ConvDesc, seed=0, dev="cuda:0"):
+    z, dy = make_wgrad_inputs(d, seed)
+    got = run_wgrad(d, z, dy, dev)
+    want = oracle.wgrad_compressed(synth.to_f64(z), synth.to_f64(dy), d.H, d.W, d.R, d.S,
+                                   d.stride, d.pad, d.k)
+    return float(np.linalg.norm(got - want) / np.linalg.norm(want)), got, want
+
+
+def wgrad_error_sampled(d: ac.ConvDesc, n_samples=512, seed=0, dev="cuda:0"):
+    """Full-size case: the checker evaluates `n_samples` entries of dW one by
+    one; the error is the relative l2 error over that sample."""
+    z, dy = make_wgrad_inputs(d, seed)
+    got = run_wgrad(d, z, dy, dev)
+    rng = np.random.default_rng(seed + 99)
+    idx = np.stack([rng.integers(0, d.C_out, n_samples), rng.integers(0, d.C_in, n_samples),
+                    rng.integers(0, d.R, n_samples), rng.integers(0, d.S, n_samples)], axis=1)
+    # always include the four corners of the tensor
+    idx[:4] = [[0, 0, 0, 0], [d.C_out - 1, d.C_in - 1, d.R - 1, d.S - 1],
+               [0, d.C_in - 1, 0, d.S - 1], [d.C_out - 1, 0, d.R - 1, 0]]
+    want = oracle.wgrad_compressed_entries(synth.to_f64(z), synth.to_f64(dy), d.H, d.W, d.R, d.S,
+                                           d.stride, d.pad, d.k, idx)
+    g = got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
+    assert np.isfinite(got).all()
+    return float(np.linalg.norm(g - want) / np.linalg.norm(want)), got

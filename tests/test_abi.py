@@ -1,0 +1,82 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports
+every symbol include/ac.h declares, and validates arguments before any launch."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def ac():
+    entry.build()
+    import paper_2409_11902_b200 as ac
+    return ac
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "ac.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ac_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(ac):
+    names = declared_functions()
+    assert {"ac_compress", "ac_conv2d_wgrad_compressed", "ac_workspace_bytes"} <= set(names)
+    L = ac.api.lib()
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in ac.h but not exported by libac.so"
+
+
+def test_status_strings(ac):
+    assert ac.status_string(0) == "AC_OK"
+    assert ac.status_string(4) == "AC_ERR_WORKSPACE_TOO_SMALL"
+    assert ac.status_string(6) == "AC_ERR_TIMEOUT"
+
+
+def test_workspace_bytes_is_host_only_and_rejects_bad_descriptors(ac):
+    good = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw")
+    assert ac.ac_workspace_bytes(good) >= 256
+    import dataclasses
+    for bad in (dict(N=0), dict(k=0), dict(C_out=-1), dict(R=40), dict(stride=(0, 1)),
+                dict(pad=(-1, 0)), dict(H=0)):
+        assert ac.ac_workspace_bytes(dataclasses.replace(good, **bad)) == 0, bad
+    assert ac.api.lib().ac_workspace_bytes(None) == 0
+
+
+def test_workspace_grows_with_the_problem_not_unbounded(ac):
+    small = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw")
+    huge = ac.ConvDesc(256, 512, 512, 56, 56, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw")
+    assert ac.ac_workspace_bytes(small) < ac.ac_workspace_bytes(huge) < (1 << 30)
+
+
+def test_calls_validate_before_launching(ac):
+    """No GPU here: every one of these must return before touching CUDA."""
+    L = ac.api.lib()
+    d = ac.ConvDesc(2, 8, 8, 8, 8, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw").c()
+    ref = ctypes.byref(d)
+    A = 0x10000  # a 16-byte aligned, never dereferenced address
+    assert L.ac_compress(ref, None, A, None, None) == ac.api.AC_ERR_INVALID_ARG
+    assert L.ac_compress(ref, A + 4, A, None, None) == ac.api.AC_ERR_MISALIGNED
+    assert L.ac_compress(ref, A, A, A + 8, None) == ac.api.AC_ERR_MISALIGNED
+    assert L.ac_compress(None, A, A, None, None) == ac.api.AC_ERR_INVALID_ARG
+    assert L.ac_conv2d_wgrad_compressed(ref, A, A, None, A, 1 << 30, None) == ac.api.AC_ERR_INVALID_ARG
+    assert L.ac_conv2d_wgrad_compressed(ref, A, A + 2, A, A, 1 << 30, None) == ac.api.AC_ERR_MISALIGNED
+    assert L.ac_conv2d_wgrad_compressed(ref, A, A, A, A, 16, None) == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
+    bad = ac.ConvDesc(2, 8, 8, 8, 8, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw").c()
+    bad.dtype = 7
+    assert L.ac_compress(ctypes.byref(bad), A, A, None, None) == ac.api.AC_ERR_INVALID_ARG
+    assert L.ac_backward_step_host(ref, A, A, A, None, A + 16, 1 << 30, None) == ac.api.AC_ERR_MISALIGNED
+    assert L.ac_backward_step_host(ref, A, A, A, None, A, 16, None) == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
+    assert L.ac_workspace_status(None, None, None) == ac.api.AC_ERR_INVALID_ARG
+
+
+def test_binding_fails_loudly_without_the_library(ac, monkeypatch):
+    monkeypatch.setattr(ac.api, "_lib", None)
+    monkeypatch.setattr(ac.api, "_LIB_PATH", "/nonexistent/libac.so")
+    with pytest.raises(ImportError):
+        ac.ac_workspace_bytes(ac.ConvDesc(1, 8, 8, 8, 8))

@@ -1,0 +1,67 @@
+"""GPU parity of ac_compress against the CPU checker (element by element)."""
+import pytest
+
+import __graft_entry__ as entry
+from helpers import TOL_Z, run_compress
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    entry.build()
+
+
+def desc(N, C, H, W, k, dtype, layout):
+    import paper_2409_11902_b200 as ac
+    return ac.ConvDesc(N, C, 1, H, W, 1, 1, (1, 1), (0, 0), k, dtype, layout)
+
+
+SHAPES = [
+    # N, C, H, W -- spans several 256-thread blocks, with ragged tails
+    (8, 64, 32, 32),     # config 1
+    (3, 64, 56, 56),     # ResNet 56x56 map
+    (2, 128, 28, 28),
+    (2, 256, 14, 14),
+    (2, 512, 7, 7),      # odd size: partial blocks on both edges
+    (2, 24, 9, 15),      # odd H and W, C a multiple of 8
+    (1, 3, 17, 23),      # stem-like: C not a multiple of the vector width
+    (1, 5, 1, 1),        # degenerate map
+]
+
+
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("k", [1, 2, 3, 4, 8])
+@pytest.mark.parametrize("shape", SHAPES)
+def test_compress_matches_checker(shape, k, dtype, layout):
+    err, _, _ = run_compress(desc(*shape, k, dtype, layout))
+    assert err <= TOL_Z[dtype], err
+
+
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+@pytest.mark.parametrize("inplace", [False, True])
+@pytest.mark.parametrize("shape", [(3, 64, 56, 56), (2, 512, 7, 7), (1, 3, 17, 23), (2, 32, 16, 64)])
+def test_fused_relu_compress(shape, inplace, k, dtype, layout):
+    err, _, _ = run_compress(desc(*shape, k, dtype, layout), fused_relu=True, inplace=inplace)
+    assert err <= TOL_Z[dtype], err
+
+
+def test_large_map_many_blocks():
+    # 64 x 128 x 64 x 64 fp32 = 128 MiB: larger than L2, > 100k thread blocks
+    for layout in ("nchw", "nhwc"):
+        err, _, _ = run_compress(desc(64, 128, 64, 64, 2, "f32", layout))
+        assert err <= TOL_Z["f32"], err
+
+
+def test_runtime_errors_are_codes():
+    import torch
+    import paper_2409_11902_b200 as ac
+    d = desc(1, 8, 8, 8, 2, "f32", "nchw")
+    x = torch.zeros(d.x_shape, device="cuda")
+    z = torch.zeros(d.z_shape, device="cuda")
+    with pytest.raises(ac.AcError) as e:
+        ac.ac_compress(d, x.data_ptr() + 4, z)
+    assert e.value.status == ac.api.AC_ERR_MISALIGNED

@@ -1,0 +1,145 @@
+"""GPU parity of ac_conv2d_wgrad_compressed against the CPU checker."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import __graft_entry__ as entry
+from helpers import TOL_DW, make_wgrad_inputs, run_wgrad, wgrad_error_full, wgrad_error_sampled
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    entry.build()
+
+
+def D(N, Ci, Co, H, W, R, S, stride, pad, k, dtype, layout):
+    import paper_2409_11902_b200 as ac
+    return ac.ConvDesc(N, Ci, Co, H, W, R, S, (stride, stride), (pad, pad), k, dtype, layout)
+
+
+SMALL = [
+    # N, Ci, Co, H, W, R, S, stride, pad, k
+    (8, 64, 64, 32, 32, 3, 3, 1, 1, 2),     # config 1
+    (2, 64, 64, 14, 14, 3, 3, 1, 1, 2),
+    (2, 128, 64, 9, 11, 3, 3, 1, 1, 2),     # odd H, W: partial pooling blocks at the padding edge
+    (2, 64, 128, 7, 7, 3, 3, 1, 1, 2),
+    (2, 64, 64, 16, 16, 3, 3, 2, 1, 2),     # stride 2 (taps collapse)
+    (2, 64, 64, 15, 15, 3, 3, 2, 1, 2),
+    (3, 128, 64, 12, 12, 1, 1, 1, 0, 2),    # pointwise
+    (3, 64, 128, 12, 12, 1, 1, 2, 0, 2),    # pointwise, stride 2
+    (2, 64, 64, 16, 16, 3, 3, 1, 1, 1),     # k = 1: uncompressed
+    (2, 64, 64, 16, 16, 3, 3, 1, 1, 4),
+    (2, 64, 64, 16, 16, 3, 3, 1, 1, 8),
+    (2, 64, 64, 13, 13, 3, 3, 1, 1, 3),     # k that divides nothing
+    (1, 3, 16, 20, 20, 7, 7, 2, 3, 2),      # stem-like
+    (2, 24, 40, 10, 10, 5, 3, 1, 2, 2),     # channels not multiples of 64, R != S
+    (1, 8, 8, 4, 4, 3, 3, 1, 1, 2),         # tiny
+    (1, 64, 64, 1, 1, 1, 1, 1, 0, 2),       # degenerate map
+]
+
+
+@pytest.mark.parametrize("layout", ["nhwc", "nchw"])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("case", SMALL)
+def test_wgrad_matches_checker(case, dtype, layout):
+    err, got, want = wgrad_error_full(D(*case, dtype, layout))
+    assert err <= TOL_DW[dtype], err
+
+
+def test_k1_equals_uncompressed_dw():
+    """k = 1: Z is X, so the result must be the ordinary weight gradient."""
+    import oracle
+    from paper_2409_11902_b200 import synth
+    d = D(2, 64, 64, 16, 16, 3, 3, 1, 1, 1, "bf16", "nhwc")
+    z, dy = make_wgrad_inputs(d)
+    got = run_wgrad(d, z, dy)
+    want = oracle.wgrad_dense(synth.to_f64(z), synth.to_f64(dy), 3, 3, (1, 1), (1, 1))
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) <= TOL_DW["bf16"]
+
+
+def test_tap_collapse_on_gpu():
+    """Stride 2, k = 2, pad 1, even H: taps 1 and 2 read the same pooled value,
+    so the two slices of dW must agree exactly (same products, same order)."""
+    d = D(2, 64, 64, 16, 16, 3, 3, 2, 1, 2, "bf16", "nhwc")
+    z, dy = make_wgrad_inputs(d)
+    got = run_wgrad(d, z, dy)
+    np.testing.assert_allclose(got[:, :, 1, :], got[:, :, 2, :], rtol=1e-5, atol=1e-7)
+    np.testing.assert_allclose(got[:, :, :, 1], got[:, :, :, 2], rtol=1e-5, atol=1e-7)
+
+
+RESNET18_STACK = [   # config 2: batch 64, bf16, k = 2 (+ the 7x7 map padded to 8x8)
+    (64, 64, 64, 56, 56), (64, 128, 128, 28, 28), (64, 256, 256, 14, 14),
+    (64, 512, 512, 7, 7), (64, 512, 512, 8, 8),
+]
+
+
+@pytest.mark.parametrize("N,Ci,Co,H,W", RESNET18_STACK)
+def test_resnet18_stack_full_size_sampled(N, Ci, Co, H, W):
+    err, _ = wgrad_error_sampled(D(N, Ci, Co, H, W, 3, 3, 1, 1, 2, "bf16", "nhwc"), n_samples=512)
+    assert err <= TOL_DW["bf16"], err
+
+
+BOTTLENECK = [  # config 3: batch 128, bf16
+    (128, 256, 64, 56, 56, 1, 1, 1, 0), (128, 64, 64, 56, 56, 3, 3, 1, 1),
+    (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
+]
+
+
+@pytest.mark.parametrize("N,Ci,Co,H,W,R,S,stride,pad", BOTTLENECK)
+def test_bottleneck_layers_full_size_sampled(N, Ci, Co, H, W, R, S, stride, pad):
+    err, _ = wgrad_error_sampled(D(N, Ci, Co, H, W, R, S, stride, pad, 2, "bf16", "nhwc"),
+                                 n_samples=256)
+    assert err <= TOL_DW["bf16"], err
+
+
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+def test_pooling_sweep_full_size_sampled(k):
+    """Config 4: N=256, 128 channels, 64x64, bf16 (1 Mi positions per entry)."""
+    err, _ = wgrad_error_sampled(D(256, 128, 128, 64, 64, 3, 3, 1, 1, k, "bf16", "nhwc"),
+                                 n_samples=96)
+    assert err <= TOL_DW["bf16"], err
+
+
+def test_errors_are_codes_not_faults():
+    import torch
+    import paper_2409_11902_b200 as ac
+    d = D(2, 64, 64, 16, 16, 3, 3, 1, 1, 2, "bf16", "nhwc")
+    z = torch.zeros(d.z_shape, dtype=torch.bfloat16, device="cuda")
+    dy = torch.zeros(d.dy_shape, dtype=torch.bfloat16, device="cuda")
+    dw = torch.zeros(d.dw_shape, device="cuda")
+    n = ac.ac_workspace_bytes(d)
+    ws = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    with pytest.raises(ac.AcError) as e:
+        ac.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws, n - 1)
+    assert e.value.status == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(ac.AcError) as e:
+        ac.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws.data_ptr() + 8, n)
+    assert e.value.status == ac.api.AC_ERR_MISALIGNED
+    ac.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws, n)
+    assert ac.ac_workspace_status(ws) == (0, 0)
+    assert not dw.any()
+
+
+def test_host_step_matches_device_calls():
+    import torch
+    import paper_2409_11902_b200 as ac
+    from paper_2409_11902_b200 import synth
+    d = D(4, 64, 64, 16, 16, 3, 3, 1, 1, 2, "bf16", "nhwc")
+    x = synth.to_layout(synth.activation(0, (d.N, d.C_in, d.H, d.W), d.dtype), d.layout).pin_memory()
+    dy = synth.to_layout(synth.grad_output(0, (d.N, d.C_out, d.Ho, d.Wo), d.dtype), d.layout).pin_memory()
+    dw_h = torch.empty(d.dw_shape, dtype=torch.float32).pin_memory()
+    z_h = torch.empty(d.z_shape, dtype=torch.bfloat16).pin_memory()
+    arena = torch.empty(ac.ac_host_step_arena_bytes(d), dtype=torch.uint8, device="cuda")
+    ac.ac_backward_step_host(d, x, dy, dw_h, z_h, arena)
+    torch.cuda.synchronize()
+    xd, dyd = x.cuda(), dy.cuda()
+    z = torch.empty(d.z_shape, dtype=torch.bfloat16, device="cuda")
+    dw = torch.empty(d.dw_shape, device="cuda")
+    ws = torch.empty(ac.ac_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+    ac.ac_compress(d, xd, z)
+    ac.ac_conv2d_wgrad_compressed(d, z, dyd, dw, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(z.cpu(), z_h) and torch.equal(dw.cpu(), dw_h)
