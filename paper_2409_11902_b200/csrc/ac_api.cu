@@ -35,13 +35,8 @@ ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o) {
 
 static inline long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
 
-WgradPlan plan_wgrad(const Dims& d) {
+WgradPlan plan_wgrad_simt(const Dims& d) {
     WgradPlan p{};
-    if (tc_supported(d)) {
-        p.path = PATH_TC;
-        plan_tc(d, &p);
-        return p;
-    }
     p.path = PATH_SIMT;
     const long long K = d.K();
     const long long J = (long long)d.Ci * d.R * d.S;
@@ -61,6 +56,16 @@ WgradPlan plan_wgrad(const Dims& d) {
     p.splits = (int)ceil_div(K, kps);
     p.bytes = kStatusBlockBytes + (p.splits > 1 ? (size_t)p.splits * dw_bytes : 0);
     return p;
+}
+
+WgradPlan plan_wgrad(const Dims& d) {
+    if (tc_supported(d)) {
+        WgradPlan p{};
+        p.path = PATH_TC;
+        plan_tc(d, &p);
+        return p;
+    }
+    return plan_wgrad_simt(d);
 }
 
 }  // namespace ac

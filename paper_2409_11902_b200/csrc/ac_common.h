@@ -49,6 +49,7 @@ struct WgradPlan {
 };
 
 WgradPlan plan_wgrad(const Dims& d);
+WgradPlan plan_wgrad_simt(const Dims& d);  // the fp32-ALU path's plan, whatever plan_wgrad picks
 
 // ---- launchers (each enqueues on `stream`, returns AC_OK or AC_ERR_CUDA) -----
 ac_status launch_compress(const Dims& d, const void* x, void* z, void* y_out, cudaStream_t stream);
