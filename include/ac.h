@@ -145,6 +145,34 @@ ac_status ac_backward_step_host(const ac_conv_desc *desc, const void *x_host,
                                 const void *dy_host, float *dw_host, void *z_host,
                                 void *arena, size_t arena_bytes, void *stream);
 
+/*
+ * The weight gradient without a workspace argument, for callers that cannot
+ * allocate device memory. (The paper has no counterpart to this call; it
+ * exists for the library's users, not for the method.)
+ *
+ * Some callers have no way to get scratch memory: they run inside a framework
+ * whose memory pool already holds the whole device, so a raw cudaMalloc fails
+ * or stalls every stream; or in a loop that must never wait on the allocator;
+ * or as a plug-in that receives tensors but no allocator. For them the scratch
+ * is a fixed array of AC_STATIC_SCRATCH_BYTES bytes of device memory that
+ * belongs to the library image: every GPU that loads the library holds it
+ * until the process ends. The call allocates and frees nothing.
+ *
+ * Computes the same dW as ac_conv2d_wgrad_compressed (same arguments z, dy,
+ * dw, same layouts, dW overwritten), always on the fp32-ALU kernel.
+ *   - Problems whose split-K scratch would exceed AC_STATIC_SCRATCH_BYTES are
+ *     refused with AC_ERR_WORKSPACE_TOO_SMALL before anything is launched.
+ *   - The first call on each device looks up the array's device address (the
+ *     device must be current). Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which still holds the last
+ *     call's partial sums: two calls that overlap on the GPU (different streams,
+ *     or different host threads without ordering) race. Issue them on one stream
+ *     or order them yourself.
+ */
+#define AC_STATIC_SCRATCH_BYTES (32u << 20)
+ac_status ac_conv2d_wgrad_compressed_static(const ac_conv_desc *desc, const void *z,
+                                            const void *dy, float *dw, void *stream);
+
 /* Static, human-readable name of a status code. */
 const char *ac_status_string(ac_status status);
 

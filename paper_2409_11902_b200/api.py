@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.ac_host_step_arena_bytes.argtypes = [dp]
         L.ac_backward_step_host.restype = ctypes.c_int
         L.ac_backward_step_host.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
+        L.ac_conv2d_wgrad_compressed_static.restype = ctypes.c_int
+        L.ac_conv2d_wgrad_compressed_static.argtypes = [dp, vp, vp, vp, vp]
         L.ac_status_string.restype = ctypes.c_char_p
         L.ac_status_string.argtypes = [ctypes.c_int]
         _lib = L
@@ -186,3 +188,13 @@ def ac_backward_step_host(desc: ConvDesc, x_host, dy_host, dw_host, z_host, aren
                                      _ptr(z_host), _ptr(arena), arena_bytes, _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_backward_step_host")
+
+
+def ac_conv2d_wgrad_compressed_static(desc: ConvDesc, z, dy, dw, stream=None) -> None:
+    """dW without a workspace argument: the scratch is a fixed array inside the
+    library (see include/ac.h). For callers that cannot allocate device memory."""
+    c = desc.c()
+    st = lib().ac_conv2d_wgrad_compressed_static(ctypes.byref(c), _ptr(z), _ptr(dy), _ptr(dw),
+                                                 _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_conv2d_wgrad_compressed_static")
