@@ -173,6 +173,28 @@ ac_status ac_backward_step_host(const ac_conv_desc *desc, const void *x_host,
 ac_status ac_conv2d_wgrad_compressed_static(const ac_conv_desc *desc, const void *z,
                                             const void *dy, float *dw, void *stream);
 
+/*
+ * How ac_conv2d_wgrad_compressed will run this problem (pure host code; for
+ * reports and tests). Returns AC_ERR_INVALID_ARG for an invalid descriptor.
+ */
+typedef struct {
+    int32_t tensor_core;     /* 1: tcgen05 kernel, 0: fp32-ALU kernel */
+    int32_t splits;          /* K-slices summed by the split-K reduction */
+    int32_t ctas;            /* CTAs of the main kernel */
+    int32_t groups;          /* tensor-core path: CTAs that share one K-slice */
+    int32_t band_rows;       /* tensor-core path: output rows per K-tile */
+    int32_t k_tile;          /* tensor-core path: positions per K-tile incl. zero fill */
+    int32_t row_pitch;       /* tensor-core path: flat row pitch Wq of the tiles */
+    int32_t stages;          /* tensor-core path: shared-memory pipeline depth */
+    int32_t smem_bytes;      /* dynamic shared memory per CTA */
+    int32_t tmem_columns;    /* tensor-memory columns allocated per CTA */
+    int32_t units_per_cta;   /* tensor-core path: accumulator tiles (128 x block_n) per CTA */
+    int32_t block_n;         /* tensor-core path: output channels per accumulator tile */
+    int32_t a_cells;         /* tensor-core path: cells per plane of the inflated input grid */
+    int32_t phases;          /* tensor-core path: stride phases held in shared memory */
+} ac_plan_info;
+ac_status ac_wgrad_plan_info(const ac_conv_desc *desc, ac_plan_info *info);
+
 /* Static, human-readable name of a status code. */
 const char *ac_status_string(ac_status status);
 

@@ -34,6 +34,12 @@ class ac_conv_desc(ctypes.Structure):
         "pad_h", "pad_w", "k", "dtype", "layout")]
 
 
+class ac_plan_info(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "tensor_core", "splits", "ctas", "groups", "band_rows", "k_tile", "row_pitch", "stages",
+        "smem_bytes", "tmem_columns", "units_per_cta", "block_n", "a_cells", "phases")]
+
+
 class AcError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -68,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.ac_backward_step_host.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
         L.ac_conv2d_wgrad_compressed_static.restype = ctypes.c_int
         L.ac_conv2d_wgrad_compressed_static.argtypes = [dp, vp, vp, vp, vp]
+        L.ac_wgrad_plan_info.restype = ctypes.c_int
+        L.ac_wgrad_plan_info.argtypes = [dp, ctypes.POINTER(ac_plan_info)]
         L.ac_status_string.restype = ctypes.c_char_p
         L.ac_status_string.argtypes = [ctypes.c_int]
         _lib = L
@@ -198,3 +206,13 @@ def ac_conv2d_wgrad_compressed_static(desc: ConvDesc, z, dy, dw, stream=None) ->
                                                  _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_conv2d_wgrad_compressed_static")
+
+
+def ac_wgrad_plan_info(desc: ConvDesc) -> dict:
+    """How the library will run this problem (host arithmetic only)."""
+    c = desc.c()
+    info = ac_plan_info()
+    st = lib().ac_wgrad_plan_info(ctypes.byref(c), ctypes.byref(info))
+    if st != AC_OK:
+        raise AcError(st, "ac_wgrad_plan_info")
+    return {n: getattr(info, n) for n, _ in ac_plan_info._fields_}

@@ -156,6 +156,24 @@ ac_status ac_backward_step_host(const ac_conv_desc* desc, const void* x_host, co
     return AC_OK;
 }
 
+ac_status ac_wgrad_plan_info(const ac_conv_desc* desc, ac_plan_info* info) {
+    Dims d;
+    if (!info) return AC_ERR_INVALID_ARG;
+    ac_status st = make_dims(desc, true, &d);
+    if (st != AC_OK) return st;
+    *info = ac_plan_info{};
+    if (tc_supported(d)) {
+        tc_plan_info(d, info);
+        return AC_OK;
+    }
+    const WgradPlan p = plan_wgrad_simt(d);
+    const long long J = (long long)d.Ci * d.R * d.S;
+    info->splits = p.splits;
+    info->ctas = (int32_t)(((J + 63) / 64) * ((d.Co + 63) / 64) * p.splits);
+    info->smem_bytes = 0;
+    return AC_OK;
+}
+
 const char* ac_status_string(ac_status status) {
     switch (status) {
         case AC_OK: return "AC_OK";

@@ -57,6 +57,7 @@ ac_status launch_wgrad_simt(const Dims& d, const WgradPlan& p, const void* z, co
                             float* dw, void* workspace, cudaStream_t stream);
 bool tc_supported(const Dims& d);
 void plan_tc(const Dims& d, WgradPlan* p);
+void tc_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_tc(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                           float* dw, void* workspace, cudaStream_t stream);
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,

@@ -80,3 +80,37 @@ def test_binding_fails_loudly_without_the_library(ac, monkeypatch):
     monkeypatch.setattr(ac.api, "_LIB_PATH", "/nonexistent/libac.so")
     with pytest.raises(ImportError):
         ac.ac_workspace_bytes(ac.ConvDesc(1, 8, 8, 8, 8))
+
+
+def test_plan_info_respects_hardware_limits(ac):
+    """Host-side planning of the tensor-core path: shared memory, tensor memory
+    and pipeline depth stay inside what one SM has, for every benchmark layer."""
+    shapes = [
+        (64, 64, 64, 56, 56, 3, 3, 1, 1), (64, 128, 128, 28, 28, 3, 3, 1, 1),
+        (64, 256, 256, 14, 14, 3, 3, 1, 1), (64, 512, 512, 7, 7, 3, 3, 1, 1),
+        (64, 512, 512, 8, 8, 3, 3, 1, 1), (128, 256, 64, 56, 56, 1, 1, 1, 0),
+        (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
+        (256, 128, 128, 64, 64, 3, 3, 1, 1), (256, 1024, 2048, 14, 14, 1, 1, 2, 0),
+        (8, 64, 64, 30, 30, 7, 7, 2, 3), (2, 192, 320, 9, 200, 3, 3, 1, 1),
+    ]
+    for N, ci, co, H, W, R, S, st, pd in shapes:
+        for k in (1, 2, 4, 8):
+            d = ac.ConvDesc(N, ci, co, H, W, R, S, (st, st), (pd, pd), k, "bf16", "nhwc")
+            i = ac.ac_wgrad_plan_info(d)
+            assert i["tensor_core"] == 1, d
+            assert 2 <= i["stages"] <= 8
+            assert i["smem_bytes"] <= 227 * 1024
+            assert i["tmem_columns"] in (32, 64, 128, 256, 512)
+            assert i["units_per_cta"] * i["block_n"] <= i["tmem_columns"]
+            assert i["k_tile"] % 16 == 0 and i["k_tile"] >= i["band_rows"] * i["row_pitch"]
+            assert i["row_pitch"] >= d.Wo
+            assert 1 <= i["splits"] <= d.N * -(-d.Ho // i["band_rows"])
+            assert i["ctas"] == i["splits"] * i["groups"]
+            want = 256 + (i["splits"] * 4 * co * ci * R * S if i["splits"] > 1 else 0)
+            assert ac.ac_workspace_bytes(d) == want
+    # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
+    for d in (ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nhwc"),
+              ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
+              ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc"),
+              ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (3, 3), (1, 1), 2, "bf16", "nhwc")):
+        assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 0
