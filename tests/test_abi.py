@@ -91,7 +91,7 @@ def test_plan_info_respects_hardware_limits(ac):
         (64, 512, 512, 8, 8, 3, 3, 1, 1), (128, 256, 64, 56, 56, 1, 1, 1, 0),
         (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
         (256, 128, 128, 64, 64, 3, 3, 1, 1), (256, 1024, 2048, 14, 14, 1, 1, 2, 0),
-        (8, 64, 64, 30, 30, 7, 7, 2, 3), (2, 192, 320, 9, 200, 3, 3, 1, 1),
+        (8, 64, 64, 30, 30, 7, 7, 2, 3), (2, 192, 320, 9, 40, 3, 3, 1, 1),
     ]
     for N, ci, co, H, W, R, S, st, pd in shapes:
         for k in (1, 2, 4, 8):
