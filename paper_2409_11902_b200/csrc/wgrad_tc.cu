@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kThreads, 1) wgrad_tc_kernel(const __grid_cons
         // ------------------------------------------------------------ producers
         const int cgh_n = ncib * p.ncgpc / 8;          // groups of 8 channel-group planes
         const int totalA = p.nph * cgh_n * p.NC * 8;
-        const int totalB = (p.BN / 8) * p.KT * 8;
+        const int totalB = (p.BN / 8) * p.KT;          // 16-byte vectors: 8 channels x 1 position
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         for (int kt = kt_begin, it = 0; kt < kt_end; ++kt, ++it) {
             const int s = it % p.stages;
