@@ -76,7 +76,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -181,14 +181,6 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     total_ms = t0.elapsed_time(t1)
-    if rank == 0:
-        # keep the sampler over a short stretch of identical extra work if the timed
-        # region was shorter than its period, so that clocks under load are seen
-        t_end = time.time() + 0.5
-        it = 0
-        while time.time() < t_end:
-            step(it); it += 1
-        torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
     if world > 1:
         t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
@@ -335,7 +327,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()

@@ -190,6 +190,26 @@ __global__ void __launch_bounds__(kThreads, 1) wgrad_tc_kernel(const __grid_cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kProducerWarps) tmem_alloc(&tmem_base_s, p.tmem_cols);
+    if (warp < kProducerWarps) {
+        // Cells past the last grid row (read by the last K steps of the last taps)
+        // and positions past the last tile row are never written again: zero them
+        // once so that they are finite (they only ever meet zeros of the other operand).
+        const int tailA = p.NC - p.GH * p.Wq, tailB = p.KT - p.hb * p.Wq;
+        const int planesA_all = (int)(p.a_stage_bytes / p.sbo_a);
+        const uint4 zero4 = make_uint4(0, 0, 0, 0);
+        for (int s = 0; s < p.stages; ++s) {
+            unsigned char* a_st = tc_smem + (size_t)s * stage_bytes;
+            unsigned char* b_st = a_st + p.a_stage_bytes;
+            for (int e = tid; e < planesA_all * tailA; e += kProducerThreads) {
+                const int pl = e / tailA, c = p.GH * p.Wq + (e - pl * tailA);
+                *reinterpret_cast<uint4*>(a_st + (size_t)pl * p.sbo_a + (size_t)c * 16) = zero4;
+            }
+            for (int e = tid; e < (p.BN / 8) * tailB; e += kProducerThreads) {
+                const int pl = e / tailB, q = p.hb * p.Wq + (e - pl * tailB);
+                *reinterpret_cast<uint4*>(b_st + (size_t)pl * p.sbo_b + (size_t)q * 16) = zero4;
+            }
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -197,10 +217,25 @@ __global__ void __launch_bounds__(kThreads, 1) wgrad_tc_kernel(const __grid_cons
 
     if (warp < kProducerWarps) {
         // ------------------------------------------------------------ producers
-        const int cgh_n = ncib * p.ncgpc / 8;          // groups of 8 channel-group planes
-        const int totalA = p.nph * cgh_n * p.NC * 8;
-        const int totalB = (p.BN / 8) * p.KT;          // 16-byte vectors: 8 channels x 1 position
+        // A K-tile is filled row by row. A "job" is one row of one plane group
+        // (8 planes = 64 channels): first the rows of the inflated input grid(s),
+        // then the rows of the output-gradient tile. A warp step covers 4 cells x
+        // 8 planes (lane = plane + 8 * cell): 128 contiguous bytes per cell from
+        // global memory, and 8 planes x 16 bytes = all 32 banks per quarter warp
+        // in shared memory (plane strides are odd multiples of 16 bytes).
+        // Steps are dealt round-robin to the warps and handled kBatch at a time:
+        // all loads of a batch are issued before its first store.
+        constexpr int kBatch = 8;
+        const int cgh_n = ncib * p.ncgpc / 8;          // plane groups of the input grid
+        const int cogh_n = p.BN / 64;                  // plane groups of the gradient tile
+        const int jobsA = p.nph * p.GH * cgh_n;
+        const int jobs = jobsA + p.hb * cogh_n;
+        const int cpr = (p.Wq + 3) >> 2;               // warp steps per row
+        const int steps = jobs * cpr;
+        const int cgl = lane & 7, jl = lane >> 3;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
+        const __nv_bfloat16* zsrc = p.z + cib0 * p.CB + cgl * 8;
+        const __nv_bfloat16* gsrc = p.dy + co0 + cgl * 8;
         for (int kt = kt_begin, it = 0; kt < kt_end; ++kt, ++it) {
             const int s = it % p.stages;
             const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
@@ -212,40 +247,48 @@ __global__ void __launch_bounds__(kThreads, 1) wgrad_tc_kernel(const __grid_cons
             const int ho0 = band * p.hb;
             unsigned char* a_st = tc_smem + (size_t)s * stage_bytes;
             unsigned char* b_st = a_st + p.a_stage_bytes;
-            // inflated, padded input grid(s): one 16-byte vector per (phase, 8 channels, cell)
-            for (int e = tid; e < totalA; e += kProducerThreads) {
-                const int cgl = e & 7;
-                int rest = e >> 3;
-                const int cell = rest % p.NC; rest /= p.NC;
-                const int cgh = rest % cgh_n;
-                const int slot = rest / cgh_n;
-                const int gi = cell / p.Wq, gj = cell - gi * p.Wq;
-                const int hx = p.sh * (ho0 + p.dr_min + gi) + p.phase_a[slot];
-                const int wx = p.sw * (p.dc_min + gj) + p.phase_b[slot];
-                const int cg = cgh * 8 + cgl;
-                uint4 v = zero4;
-                if (gi < p.GH && hx >= 0 && hx < p.H && wx >= 0 && wx < p.W) {
-                    const long long off =
-                        (((long long)n * p.Hp + hx / p.k) * p.Wp + wx / p.k) * p.Ci + cib0 * p.CB + cg * 8;
-                    v = __ldg(reinterpret_cast<const uint4*>(p.z + off));
+            int job = warp / cpr, chunk = warp - job * cpr;     // step `warp`, then += kProducerWarps
+            for (int st0 = warp; st0 < steps; st0 += kProducerWarps * kBatch) {
+                uint4 v[kBatch];
+                unsigned char* dst[kBatch];
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b) {
+                    dst[b] = nullptr;
+                    v[b] = zero4;
+                    if (st0 + b * kProducerWarps < steps) {
+                        const int gj = chunk * 4 + jl;
+                        const __nv_bfloat16* src = nullptr;
+                        if (job < jobsA) {
+                            const int slot = job / (p.GH * cgh_n);
+                            const int rem = job - slot * (p.GH * cgh_n);
+                            const int gi = rem / cgh_n, cgh = rem - gi * cgh_n;
+                            const int hx = p.sh * (ho0 + p.dr_min + gi) + p.phase_a[slot];
+                            const int wx = p.sw * (p.dc_min + gj) + p.phase_b[slot];
+                            if (gj < p.Wq) {
+                                dst[b] = a_st + (size_t)slot * p.ph_bytes +
+                                         (size_t)(cgh * 8 + cgl) * p.sbo_a + (size_t)(gi * p.Wq + gj) * 16;
+                                if (hx >= 0 && hx < p.H && wx >= 0 && wx < p.W)
+                                    src = zsrc + (((long long)n * p.Hp + hx / p.k) * p.Wp + wx / p.k) * p.Ci +
+                                          cgh * 64;
+                            }
+                        } else {
+                            const int jb = job - jobsA;
+                            const int i = jb / cogh_n, cogh = jb - i * cogh_n;
+                            const int ho = ho0 + i;
+                            if (gj < p.Wq) {
+                                dst[b] = b_st + (size_t)(cogh * 8 + cgl) * p.sbo_b + (size_t)(i * p.Wq + gj) * 16;
+                                if (ho < p.Ho && gj < p.Wo)
+                                    src = gsrc + (((long long)n * p.Ho + ho) * p.Wo + gj) * p.Co + cogh * 64;
+                            }
+                        }
+                        if (src) v[b] = __ldg(reinterpret_cast<const uint4*>(src));
+                    }
+                    chunk += kProducerWarps;
+                    while (chunk >= cpr) { chunk -= cpr; ++job; }
                 }
-                *reinterpret_cast<uint4*>(a_st + (size_t)slot * p.ph_bytes + (size_t)cg * p.sbo_a +
-                                          (size_t)cell * 16) = v;
-            }
-            // output-gradient tile, flat positions with pitch Wq, zero in the surplus
-            for (int e = tid; e < totalB; e += kProducerThreads) {
-                const int cogl = e & 7;
-                const int rest = e >> 3;
-                const int q = rest % p.KT;
-                const int cog = (rest / p.KT) * 8 + cogl;
-                const int i = q / p.Wq, wo = q - i * p.Wq;
-                const int ho = ho0 + i;
-                uint4 v = zero4;
-                if (i < p.hb && ho < p.Ho && wo < p.Wo) {
-                    const long long off = (((long long)n * p.Ho + ho) * p.Wo + wo) * p.Co + co0 + cog * 8;
-                    v = __ldg(reinterpret_cast<const uint4*>(p.dy + off));
-                }
-                *reinterpret_cast<uint4*>(b_st + (size_t)cog * p.sbo_b + (size_t)q * 16) = v;
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b)
+                    if (dst[b]) *reinterpret_cast<uint4*>(dst[b]) = v[b];
             }
             fence_proxy_async_smem();   // generic-proxy stores -> visible to the tensor core's reads
             mbar_arrive(&full_bar[s]);
