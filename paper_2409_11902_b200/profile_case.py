@@ -1,0 +1,61 @@
+"""Runs one layer of the hot path a few times on cuda:0: the small, bounded
+workload that profiler captures (ncu) are taken on.
+
+    python -m paper_2409_11902_b200.profile_case --layer 128ch_28x28 --batch 16 --iters 3
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import api, synth
+
+LAYERS = {
+    # name: (C_in, C_out, H, W, R, S, stride, pad)
+    "64ch_56x56": (64, 64, 56, 56, 3, 3, 1, 1),
+    "128ch_28x28": (128, 128, 28, 28, 3, 3, 1, 1),
+    "256ch_14x14": (256, 256, 14, 14, 3, 3, 1, 1),
+    "512ch_8x8": (512, 512, 8, 8, 3, 3, 1, 1),
+    "128ch_64x64": (128, 128, 64, 64, 3, 3, 1, 1),
+    "128ch_56x56_s2": (128, 128, 56, 56, 3, 3, 2, 1),
+    "256to64_1x1_56x56": (256, 64, 56, 56, 1, 1, 1, 0),
+}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--layer", default="128ch_28x28", choices=sorted(LAYERS))
+    ap.add_argument("--batch", type=int, default=16)
+    ap.add_argument("--k", type=int, default=2)
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--dtype", default="bf16")
+    ap.add_argument("--layout", default="nhwc")
+    ap.add_argument("--relu", action="store_true", help="use the fused ReLU+compress form")
+    a = ap.parse_args()
+    ci, co, H, W, R, S, st, pd = LAYERS[a.layer]
+    d = api.ConvDesc(a.batch, ci, co, H, W, R, S, (st, st), (pd, pd), a.k, a.dtype, a.layout)
+    dev = torch.device("cuda:0")
+    x = synth.to_layout(synth.activation(0, (d.N, ci, H, W), a.dtype), a.layout).to(dev)
+    dy = synth.to_layout(synth.grad_output(0, (d.N, co, d.Ho, d.Wo), a.dtype), a.layout).to(dev)
+    z = torch.empty(d.z_shape, dtype=d.torch_dtype, device=dev)
+    y = torch.empty_like(x) if a.relu else None
+    dw = torch.empty(d.dw_shape, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)
+    print("plan:", api.ac_wgrad_plan_info(d))
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    for it in range(a.iters):
+        e0.record()
+        api.ac_compress(d, x, z, y)
+        e1.record()
+        api.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws)
+        e2.record()
+        torch.cuda.synchronize()
+        st_, detail = api.ac_workspace_status(ws)
+        assert st_ == 0, (st_, detail)
+        print(f"iter {it}: compress {e0.elapsed_time(e1) * 1e3:.1f} us, wgrad {e1.elapsed_time(e2) * 1e3:.1f} us "
+              f"({d.flops / e1.elapsed_time(e2) / 1e9:.1f} TFLOP/s)")
+
+
+if __name__ == "__main__":
+    main()
