@@ -178,7 +178,8 @@ ac_status ac_conv2d_wgrad_compressed_static(const ac_conv_desc *desc, const void
  * reports and tests). Returns AC_ERR_INVALID_ARG for an invalid descriptor.
  */
 typedef struct {
-    int32_t tensor_core;     /* 1: tcgen05 kernel, 0: fp32-ALU kernel */
+    int32_t tensor_core;     /* 2: TMA-fed tcgen05 kernel, 1: tcgen05 kernel with inflating
+                                producer warps, 0: fp32-ALU kernel */
     int32_t splits;          /* K-slices summed by the split-K reduction */
     int32_t ctas;            /* CTAs of the main kernel */
     int32_t groups;          /* tensor-core path: CTAs that share one K-slice */
@@ -191,7 +192,8 @@ typedef struct {
     int32_t units_per_cta;   /* tensor-core path: accumulator tiles (128 x block_n) per CTA */
     int32_t block_n;         /* tensor-core path: output channels per accumulator tile */
     int32_t a_cells;         /* tensor-core path: cells per plane of the inflated input grid */
-    int32_t phases;          /* tensor-core path: stride phases held in shared memory */
+    int32_t phases;          /* tensor-core path: stride phases (kernel 1) or output classes
+                                (kernel 2) per K-tile */
 } ac_plan_info;
 ac_status ac_wgrad_plan_info(const ac_conv_desc *desc, ac_plan_info *info);
 

@@ -59,6 +59,11 @@ WgradPlan plan_wgrad_simt(const Dims& d) {
 }
 
 WgradPlan plan_wgrad(const Dims& d) {
+    if (tc2_supported(d, nullptr)) {
+        WgradPlan p{};
+        plan_tc2(d, &p);
+        return p;
+    }
     if (tc_supported(d)) {
         WgradPlan p{};
         p.path = PATH_TC;
@@ -102,6 +107,7 @@ ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, co
     if (workspace_bytes < p.bytes) return AC_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
+    if (p.path == PATH_TC2) return launch_wgrad_tc2(d, p, z, dy, dw, workspace, s);
     if (p.path == PATH_TC) return launch_wgrad_tc(d, p, z, dy, dw, workspace, s);
     return launch_wgrad_simt(d, p, z, dy, dw, workspace, s);
 }
@@ -162,6 +168,10 @@ ac_status ac_wgrad_plan_info(const ac_conv_desc* desc, ac_plan_info* info) {
     ac_status st = make_dims(desc, true, &d);
     if (st != AC_OK) return st;
     *info = ac_plan_info{};
+    if (tc2_supported(d, nullptr)) {
+        tc2_plan_info(d, info);
+        return AC_OK;
+    }
     if (tc_supported(d)) {
         tc_plan_info(d, info);
         return AC_OK;

@@ -33,7 +33,7 @@ ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* out);
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---- wgrad planning (pure host arithmetic; decides kernel and split-K) ------
-enum WgradPath { PATH_SIMT = 0, PATH_TC = 1 };
+enum WgradPath { PATH_SIMT = 0, PATH_TC = 1, PATH_TC2 = 2 };
 
 struct WgradPlan {
     int path;        // WgradPath
@@ -60,6 +60,12 @@ void plan_tc(const Dims& d, WgradPlan* p);
 void tc_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_tc(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                           float* dw, void* workspace, cudaStream_t stream);
+// TMA-fed tensor-core kernel (no inflation in shared memory); k_eff = useful / issued K
+bool tc2_supported(const Dims& d, double* k_eff);
+void plan_tc2(const Dims& d, WgradPlan* p);
+void tc2_plan_info(const Dims& d, ac_plan_info* info);
+ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
+                           float* dw, void* workspace, cudaStream_t stream);
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
                                cudaStream_t stream);
 

@@ -1,0 +1,444 @@
+// Compressed weight gradient on tcgen05 tensor cores, fed entirely by TMA.
+//
+// Same contraction as wgrad_tc.cu,
+//   dW[co,r,s,ci] = sum_{n,ho,wo} dY[n,ho,wo,co] * Xt[n, ho*sh-ph+r, wo*sw-pw+s, ci],
+// Xt = Z inflated by k (Section 4 of the paper), but the inflation is folded
+// into the addressing instead of being written out in shared memory.
+//
+// Take k = 2, stride 1. Xt[h][w] = Z[h/2][w/2], so for the outputs with
+// ho = 2i + a, wo = 2j + b (one "class" (a,b) of the four parity classes) tap
+// (r,s) reads Z[i + u][j + v] with u = floor((a - ph + r)/2), v = floor((b - pw
+// + s)/2): a constant shift of the COMPACT Z tile. In general, when the strides
+// divide k and k divides H and W, the outputs split into (k/sh)*(k/sw) classes
+// and each (class, tap) pair is a shift (u,v) of Z. Zero padding falls out of
+// the tile bounds: x < 0 or x >= H  <=>  z < 0 or z >= H/k.
+//
+// So per K-tile (one band of class rows of one image):
+//   A operand: the Z halo tile, loaded by TMA, one 8-channel plane per copy,
+//              into the un-swizzled MN-major layout [plane][cell][8 channels];
+//              a (class, tap) pair only moves the descriptor's start address.
+//   B operand: for each class, the de-interleaved dY tile, loaded by TMA through
+//              a per-class tensor map (strides c_w*Co and c_h*Wo*Co), 128-byte
+//              swizzled, rows past the class's extent zero-filled by TMA.
+//   Both use the same flat row pitch Wzq, which is what makes a tap a pure shift.
+// One thread issues the TMA copies, one thread issues tcgen05.mma, four warps
+// drain the accumulators from tensor memory at the end. K is split over CTAs.
+#include <cuda.h>
+
+#include "ac_common.h"
+#include "tc_ptx.cuh"
+#include "tc_units.h"
+
+namespace ac {
+namespace {
+
+using namespace tc;
+
+constexpr int kThreads2 = 192;        // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int kMaxUnits2 = 8;
+constexpr int kMaxClasses = 16;
+constexpr int kSlotsA = 2;
+constexpr int kMaxSlotsB = 8;
+constexpr uint32_t kSmemBudget2 = 220 * 1024;
+
+struct Tc2Params {
+    CUtensorMap tmA;                  // Z as (Ci, Wp, Hp, N)
+    CUtensorMap tmB[kMaxClasses];     // dY, one strided view per class: (Co, J_b, I_a, N)
+    float* out;
+    uint32_t* status;
+    int Ci, Co, R, S, sh, sw, ph, pw, k;
+    int c_h, c_w, ncls;
+    int umin, vmin;
+    int Wzq, Ic, bands, KT, ksteps, rowsA;
+    int CB, ncgpc, ncib_total, BN, nchunks;
+    int taps_per_group, ntapgroups, cibs_per_group, ncibgroups, groups, splits, ktiles;
+    int slotsB;
+    uint32_t a_slot_bytes, b_slot_bytes, b_chunk_bytes, sbo_a, a_box_bytes, b_box_bytes, tmem_cols;
+    long long dw_elems;
+};
+
+extern __shared__ __align__(1024) unsigned char tc2_smem[];
+
+__device__ __forceinline__ void flag_timeout(int* abort_s, uint32_t* status, uint32_t code) {
+    if (atomicExch(abort_s, 1) == 0) {
+        status[1] = code;
+        atomicExch(&status[0], 1u);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_constant__ Tc2Params p) {
+    __shared__ uint64_t fullA[kSlotsA], emptyA[kSlotsA];
+    __shared__ uint64_t fullB[kMaxSlotsB], emptyB[kMaxSlotsB];
+    __shared__ uint64_t done_bar;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    __shared__ uint32_t aoff_tab[kMaxClasses][kMaxUnits2];   // A start offset of (class, unit)
+    volatile int* abort_flag = &abort_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int group = blockIdx.x % p.groups, split = blockIdx.x / p.groups;
+    const int tg = group % p.ntapgroups;
+    const int cibg = (group / p.ntapgroups) % p.ncibgroups;
+    const int cob = group / (p.ntapgroups * p.ncibgroups);
+    const int RS = p.R * p.S;
+    const int tap0 = tg * p.taps_per_group;
+    const int ntap = min(p.taps_per_group, RS - tap0);
+    const int cib0 = cibg * p.cibs_per_group;
+    const int ncib = min(p.cibs_per_group, p.ncib_total - cib0);
+    const int nunits = ncib * ntap;
+    const int co0 = cob * p.BN;
+    const int kt_begin = (int)((long long)p.ktiles * split / p.splits);
+    const int kt_end = (int)((long long)p.ktiles * (split + 1) / p.splits);
+    // 1024-byte aligned tile area: A slots first, then B slots
+    const uint32_t smem_base = (smem_u32(tc2_smem) + 1023u) & ~1023u;
+    unsigned char* smem_gen = tc2_smem + (smem_base - smem_u32(tc2_smem));
+    const uint32_t a_base = smem_base, b_base = smem_base + kSlotsA * p.a_slot_bytes;
+
+    // Everything the MMAs may read but no copy ever writes (the cells behind the
+    // last tile row, unused planes) must be finite: zero the whole area once.
+    {
+        const uint32_t total16 = (kSlotsA * p.a_slot_bytes + p.slotsB * p.b_slot_bytes) / 16;
+        const uint4 zero4 = make_uint4(0, 0, 0, 0);
+        for (uint32_t e = tid; e < total16; e += kThreads2) reinterpret_cast<uint4*>(smem_gen)[e] = zero4;
+        fence_proxy_async_smem();
+    }
+    if (tid < p.ncls * kMaxUnits2) {
+        const int cls = tid / kMaxUnits2, u = tid % kMaxUnits2;
+        uint32_t off = 0;
+        if (u < nunits) {
+            const int cl = u / ntap, t = u - cl * ntap;
+            const int tap = tap0 + t, r = tap / p.S, sx = tap - r * p.S;
+            const int a = cls / p.c_w, b = cls - a * p.c_w;
+            const int uu = floor_div_i(p.sh * a - p.ph + r, p.k) - p.umin;
+            const int vv = floor_div_i(p.sw * b - p.pw + sx, p.k) - p.vmin;
+            off = (uint32_t)(cl * p.ncgpc) * p.sbo_a + (uint32_t)(uu * p.Wzq + vv) * 16u;
+        }
+        aoff_tab[cls][u] = off;
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], 1); }
+        for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], 1); }
+        mbar_init(&done_bar, 1);
+        abort_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tmap(&p.tmA);
+        for (int c = 0; c < p.ncls; ++c) prefetch_tmap(&p.tmB[c]);
+    }
+    if (warp == 1) tmem_alloc(&tmem_base_s, p.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    if (warp == 0 && lane == 0) {
+        // ---------------------------------------------------------- TMA producer
+        const int nplanes = ncib * p.ncgpc;
+        int tb = 0;
+        bool ok = true;
+        for (int kt = kt_begin, ta = 0; kt < kt_end && ok; ++kt, ++ta) {
+            const int sa = ta % kSlotsA;
+            if (ta >= kSlotsA && !mbar_wait(&emptyA[sa], ((ta / kSlotsA) & 1) ^ 1, abort_flag)) {
+                flag_timeout(&abort_s, p.status, 0x100u + sa);
+                break;
+            }
+            const int n = kt / p.bands, band = kt - n * p.bands;
+            const int i0 = band * p.Ic;
+            mbar_arrive_expect_tx(&fullA[sa], (uint32_t)nplanes * p.a_box_bytes);
+            const uint32_t a_slot = a_base + sa * p.a_slot_bytes;
+            for (int pl = 0; pl < nplanes; ++pl)
+                tma_load_4d(a_slot + pl * p.sbo_a, &p.tmA, &fullA[sa], cib0 * p.CB + pl * 8, p.vmin,
+                            i0 + p.umin, n);
+            for (int cls = 0; cls < p.ncls; ++cls, ++tb) {
+                const int sb = tb % p.slotsB;
+                if (tb >= p.slotsB && !mbar_wait(&emptyB[sb], ((tb / p.slotsB) & 1) ^ 1, abort_flag)) {
+                    flag_timeout(&abort_s, p.status, 0x180u + sb);
+                    ok = false;
+                    break;
+                }
+                mbar_arrive_expect_tx(&fullB[sb], (uint32_t)p.nchunks * p.b_box_bytes);
+                const uint32_t b_slot = b_base + sb * p.b_slot_bytes;
+                for (int c = 0; c < p.nchunks; ++c)
+                    tma_load_4d(b_slot + c * p.b_chunk_bytes, &p.tmB[cls], &fullB[sb], co0 + 64 * c, 0, i0, n);
+            }
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ----------------------------------------------------------- MMA issuer
+        const uint32_t idesc = make_idesc(p.BN);
+        const uint32_t a_hi = desc_hi(p.sbo_a, 0);           // un-swizzled
+        const uint32_t b_hi = desc_hi(1024, 2);              // 128-byte swizzle, 8 rows per atom
+        int tb = 0;
+        bool ok = true;
+        for (int kt = kt_begin, ta = 0; kt < kt_end && ok; ++kt, ++ta) {
+            const int sa = ta % kSlotsA;
+            if (!mbar_wait(&fullA[sa], (ta / kSlotsA) & 1, abort_flag)) {
+                flag_timeout(&abort_s, p.status, 0x200u + sa);
+                ok = false;
+                break;
+            }
+            const uint32_t a_lo0 = desc_lo(a_base + sa * p.a_slot_bytes, 128);
+            for (int cls = 0; cls < p.ncls; ++cls, ++tb) {
+                const int sb = tb % p.slotsB;
+                if (!mbar_wait(&fullB[sb], (tb / p.slotsB) & 1, abort_flag)) {
+                    flag_timeout(&abort_s, p.status, 0x280u + sb);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t b_lo0 = desc_lo(b_base + sb * p.b_slot_bytes, p.b_chunk_bytes);
+                const uint32_t first = (ta | cls) == 0 ? 0u : 1u;
+                for (int u = 0; u < nunits; ++u) {
+                    uint32_t a_lo = a_lo0 + (aoff_tab[cls][u] >> 4);
+                    uint32_t b_lo = b_lo0;
+                    const uint32_t dcol = tmem_base + (uint32_t)u * p.BN;
+                    mma_bf16_words(dcol, a_lo, a_hi, b_lo, b_hi, idesc, first);
+                    for (int kk = 1; kk < p.ksteps; ++kk) {
+                        a_lo += 16;    // 16 cells x 16 bytes
+                        b_lo += 128;   // 16 rows x 128 bytes
+                        mma_bf16_words(dcol, a_lo, a_hi, b_lo, b_hi, idesc, 1u);
+                    }
+                }
+                mma_commit(&emptyB[sb]);
+            }
+            if (ok) mma_commit(&emptyA[sa]);
+        }
+        if (ok) mma_commit(&done_bar);
+    }
+    __syncwarp();
+
+    // ---------------------------------------------------------------- epilogue
+    if (warp >= 2) {
+        bool ok = mbar_wait(&done_bar, 0, abort_flag);
+        if (!ok) flag_timeout(&abort_s, p.status, 0x300u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc_fence_after();
+            const int quarter = warp & 3;            // the TMEM lanes this warp may read
+            const int m = quarter * 32 + lane;       // accumulator row
+            float* dst = p.out + (long long)split * p.dw_elems;
+            int u = 0;
+            for (int cl = 0; cl < ncib; ++cl) {
+                const int ci = (cib0 + cl) * p.CB + m;
+                for (int t = 0; t < ntap; ++t, ++u) {
+                    const int tap = tap0 + t;
+                    for (int c0 = 0; c0 < p.BN; c0 += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(u * p.BN + c0), r);
+                        if (m < p.CB) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const long long o = ((long long)(co0 + c0 + j) * RS + tap) * p.Ci + ci;
+                                dst[o] = __uint_as_float(r[j]);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
+}
+
+// ------------------------------------------------------------------ host side
+struct Tc2Geom {
+    Tc2Params p;
+    uint32_t smem_bytes;
+    int uspan, vspan;
+    double k_eff;
+    bool ok;
+};
+
+Tc2Geom make_geom2(const Dims& d) {
+    Tc2Geom g{};
+    Tc2Params& p = g.p;
+    g.ok = false;
+    if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
+    if (d.k % d.sh != 0 || d.k % d.sw != 0) return g;      // class rows advance Z by exactly one row
+    if (d.H % d.k != 0 || d.W % d.k != 0) return g;        // padding <=> outside the Z tile
+    if (d.R * d.S > 64 || d.R > 16 || d.S > 16) return g;
+    const UnitPlan up = plan_units(d.Ci, d.Co, d.R * d.S, kMaxUnits2);
+    if (!up.ok) return g;
+    p.c_h = d.k / d.sh; p.c_w = d.k / d.sw;
+    p.ncls = p.c_h * p.c_w;
+    if (p.ncls > kMaxClasses) return g;
+    if (d.Ho < p.c_h || d.Wo < p.c_w) return g;            // every class has at least one output
+    p.Ci = d.Ci; p.Co = d.Co; p.R = d.R; p.S = d.S; p.sh = d.sh; p.sw = d.sw; p.ph = d.ph; p.pw = d.pw;
+    p.k = d.k;
+    p.dw_elems = d.dw_elems();
+    int umin = 1 << 30, umax = -(1 << 30), vmin = 1 << 30, vmax = -(1 << 30);
+    for (int a = 0; a < p.c_h; ++a)
+        for (int r = 0; r < d.R; ++r) {
+            const int u = floor_div_i(d.sh * a - d.ph + r, d.k);
+            umin = u < umin ? u : umin; umax = u > umax ? u : umax;
+        }
+    for (int b = 0; b < p.c_w; ++b)
+        for (int s = 0; s < d.S; ++s) {
+            const int v = floor_div_i(d.sw * b - d.pw + s, d.k);
+            vmin = v < vmin ? v : vmin; vmax = v > vmax ? v : vmax;
+        }
+    p.umin = umin; p.vmin = vmin;
+    g.uspan = umax - umin; g.vspan = vmax - vmin;
+    const int I = (d.Ho + p.c_h - 1) / p.c_h, Jc = (d.Wo + p.c_w - 1) / p.c_w;
+    p.Wzq = Jc + g.vspan;
+    if (p.Wzq > 256) return g;
+    p.CB = up.CB; p.ncgpc = up.ncgpc; p.ncib_total = up.ncib_total; p.BN = up.BN;
+    p.nchunks = up.BN / 64;
+    p.taps_per_group = up.taps_per_group; p.ntapgroups = up.ntapgroups;
+    p.cibs_per_group = up.cibs_per_group; p.ncibgroups = up.ncibgroups; p.groups = up.groups;
+    p.tmem_cols = up.tmem_cols;
+
+    int best_Ic = 0, best_sb = 0;
+    double best_eff = -1.0;
+    for (int want = 3; want >= 2 && best_Ic == 0; --want) {
+        for (int Ic = 1; Ic <= I; ++Ic) {
+            if (Ic + g.uspan > 256) break;
+            const int KT = (Ic * p.Wzq + 15) / 16 * 16;
+            const int NCa = (KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
+            if ((uint32_t)NCa * 16 >= (1u << 18) || (uint32_t)KT * 128 >= (1u << 18)) break;
+            const uint32_t a_slot = ((uint32_t)up.planesA * NCa * 16 + 1023) / 1024 * 1024;
+            const uint32_t b_slot = (uint32_t)p.nchunks * KT * 128;
+            if (kSlotsA * a_slot + want * b_slot > kSmemBudget2) break;
+            int sb = (int)((kSmemBudget2 - kSlotsA * a_slot) / b_slot);
+            if (sb > kMaxSlotsB) sb = kMaxSlotsB;
+            const int bands = (I + Ic - 1) / Ic;
+            const double eff = (double)d.Ho * d.Wo / ((double)bands * p.ncls * KT);
+            if (eff > best_eff + 1e-9 || (eff > best_eff - 1e-9 && Ic > best_Ic)) {
+                best_eff = eff; best_Ic = Ic; best_sb = sb;
+            }
+        }
+    }
+    if (best_Ic == 0) return g;
+    p.Ic = best_Ic;
+    p.bands = (I + p.Ic - 1) / p.Ic;
+    p.KT = (p.Ic * p.Wzq + 15) / 16 * 16;
+    p.ksteps = p.KT / 16;
+    p.rowsA = p.Ic + g.uspan;
+    const int NCa = (p.KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
+    p.sbo_a = (uint32_t)NCa * 16;
+    p.a_slot_bytes = ((uint32_t)up.planesA * p.sbo_a + 1023) / 1024 * 1024;
+    p.b_chunk_bytes = (uint32_t)p.KT * 128;
+    p.b_slot_bytes = (uint32_t)p.nchunks * p.b_chunk_bytes;
+    p.a_box_bytes = 16u * p.Wzq * p.rowsA;
+    p.b_box_bytes = 128u * p.Wzq * p.Ic;
+    p.slotsB = best_sb;
+    g.k_eff = best_eff;
+    const long long ktiles = (long long)d.N * p.bands;
+    if (ktiles >= (1ll << 30)) return g;
+    p.ktiles = (int)ktiles;
+    int splits = kNumSMs / p.groups;
+    if (splits < 1) splits = 1;
+    if (splits > p.ktiles) splits = p.ktiles;
+    p.splits = splits;
+    g.smem_bytes = kSlotsA * p.a_slot_bytes + p.slotsB * p.b_slot_bytes + 1024;
+    if (g.smem_bytes < 120 * 1024) g.smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
+    g.ok = true;
+    return g;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+    }
+    return fn;
+}
+
+}  // namespace
+
+bool tc2_supported(const Dims& d, double* k_eff) {
+    const Tc2Geom g = make_geom2(d);
+    if (g.ok && k_eff) *k_eff = g.k_eff;
+    return g.ok;
+}
+
+void plan_tc2(const Dims& d, WgradPlan* pl) {
+    const Tc2Geom g = make_geom2(d);
+    pl->path = PATH_TC2;
+    pl->splits = g.p.splits;
+    pl->tc_band = g.p.Ic * g.p.c_h;
+    pl->tc_groups = g.p.groups;
+    pl->tc_ktiles = g.p.ktiles;
+    pl->tc_stages = g.p.slotsB;
+    pl->bytes = kStatusBlockBytes + (g.p.splits > 1 ? (size_t)g.p.splits * d.dw_elems() * 4 : 0);
+}
+
+void tc2_plan_info(const Dims& d, ac_plan_info* info) {
+    const Tc2Geom g = make_geom2(d);
+    info->tensor_core = 2;
+    info->splits = g.p.splits;
+    info->ctas = g.p.splits * g.p.groups;
+    info->groups = g.p.groups;
+    info->band_rows = g.p.Ic * g.p.c_h;
+    info->k_tile = g.p.KT;
+    info->row_pitch = g.p.Wzq;
+    info->stages = g.p.slotsB;
+    info->smem_bytes = (int32_t)g.smem_bytes;
+    info->tmem_columns = (int32_t)g.p.tmem_cols;
+    info->units_per_cta = g.p.cibs_per_group * g.p.taps_per_group;
+    info->block_n = g.p.BN;
+    info->a_cells = (int32_t)(g.p.sbo_a / 16);
+    info->phases = g.p.ncls;
+}
+
+ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, const void* dy,
+                           float* dw, void* workspace, cudaStream_t stream) {
+    Tc2Geom g = make_geom2(d);
+    if (!g.ok) return AC_ERR_UNSUPPORTED;
+    Tc2Params& p = g.p;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return AC_ERR_CUDA;
+    {   // Z viewed as (Ci, Wp, Hp, N); one copy brings 8 channels of a (rows x Wzq) window
+        const cuuint64_t dims[4] = {(cuuint64_t)d.Ci, (cuuint64_t)d.Wp, (cuuint64_t)d.Hp, (cuuint64_t)d.N};
+        const cuuint64_t strides[3] = {(cuuint64_t)d.Ci * 2, (cuuint64_t)d.Wp * d.Ci * 2,
+                                       (cuuint64_t)d.Hp * d.Wp * d.Ci * 2};
+        const cuuint32_t box[4] = {8, (cuuint32_t)p.Wzq, (cuuint32_t)p.rowsA, 1};
+        const cuuint32_t es[4] = {1, 1, 1, 1};
+        if (enc(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(z), dims, strides, box, es,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return AC_ERR_CUDA;
+    }
+    for (int a = 0; a < p.c_h; ++a)
+        for (int b = 0; b < p.c_w; ++b) {
+            // class (a,b): outputs ho = c_h*i + a, wo = c_w*j + b
+            const int Ia = (d.Ho - a + p.c_h - 1) / p.c_h, Jb = (d.Wo - b + p.c_w - 1) / p.c_w;
+            const cuuint64_t dims[4] = {(cuuint64_t)d.Co, (cuuint64_t)Jb, (cuuint64_t)Ia, (cuuint64_t)d.N};
+            const cuuint64_t strides[3] = {(cuuint64_t)p.c_w * d.Co * 2, (cuuint64_t)p.c_h * d.Wo * d.Co * 2,
+                                           (cuuint64_t)d.Ho * d.Wo * d.Co * 2};
+            const cuuint32_t box[4] = {64, (cuuint32_t)p.Wzq, (cuuint32_t)p.Ic, 1};
+            const cuuint32_t es[4] = {1, 1, 1, 1};
+            char* base = static_cast<char*>(const_cast<void*>(dy)) + ((size_t)a * d.Wo + b) * d.Co * 2;
+            if (enc(&p.tmB[a * p.c_w + b], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return AC_ERR_CUDA;
+        }
+    p.status = static_cast<uint32_t*>(workspace);
+    float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBlockBytes);
+    p.out = p.splits > 1 ? partials : dw;
+    static bool attr_set = false;
+    if (!attr_set) {
+        AC_CUDA_TRY(cudaFuncSetAttribute(wgrad_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(kSmemBudget2 + 1024)));
+        attr_set = true;
+    }
+    wgrad_tc2_kernel<<<p.groups * p.splits, kThreads2, g.smem_bytes, stream>>>(p);
+    AC_CUDA_TRY(cudaGetLastError());
+    if (p.splits > 1) return launch_splitk_reduce(partials, p.splits, p.dw_elems, dw, stream);
+    (void)pl;
+    return AC_OK;
+}
+
+}  // namespace ac

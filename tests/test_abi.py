@@ -97,13 +97,20 @@ def test_plan_info_respects_hardware_limits(ac):
         for k in (1, 2, 4, 8):
             d = ac.ConvDesc(N, ci, co, H, W, R, S, (st, st), (pd, pd), k, "bf16", "nhwc")
             i = ac.ac_wgrad_plan_info(d)
-            assert i["tensor_core"] == 1, d
+            assert i["tensor_core"] in (1, 2), d
             assert 2 <= i["stages"] <= 8
             assert i["smem_bytes"] <= 227 * 1024
             assert i["tmem_columns"] in (32, 64, 128, 256, 512)
             assert i["units_per_cta"] * i["block_n"] <= i["tmem_columns"]
-            assert i["k_tile"] % 16 == 0 and i["k_tile"] >= i["band_rows"] * i["row_pitch"]
-            assert i["row_pitch"] >= d.Wo
+            assert i["k_tile"] % 16 == 0
+            if i["tensor_core"] == 1:
+                assert i["k_tile"] >= i["band_rows"] * i["row_pitch"]
+                assert i["row_pitch"] >= d.Wo
+            else:   # per class: (band_rows / c_h) class rows of row_pitch >= Wo / c_w positions
+                c_h, c_w = k // st, k // st
+                assert i["phases"] == c_h * c_w
+                assert i["k_tile"] >= (i["band_rows"] // c_h) * i["row_pitch"]
+                assert i["row_pitch"] >= -(-d.Wo // c_w)
             assert 1 <= i["splits"] <= d.N * -(-d.Ho // i["band_rows"])
             assert i["ctas"] == i["splits"] * i["groups"]
             want = 256 + (i["splits"] * 4 * co * ci * R * S if i["splits"] > 1 else 0)
