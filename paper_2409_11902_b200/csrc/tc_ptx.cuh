@@ -148,5 +148,16 @@ __device__ __forceinline__ void mma_bf16_words(uint32_t d_tmem, uint32_t a_lo, u
         : "memory");
 }
 
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 }  // namespace tc
 }  // namespace ac

@@ -94,12 +94,27 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     unsigned char* smem_gen = tc2_smem + (smem_base - smem_u32(tc2_smem));
     const uint32_t a_base = smem_base, b_base = smem_base + kSlotsA * p.a_slot_bytes;
 
-    // Everything the MMAs may read but no copy ever writes (the cells behind the
-    // last tile row, unused planes) must be finite: zero the whole area once.
+    // Everything the MMAs may read but no copy ever writes must be finite (it only
+    // ever meets zeros of the other operand, or feeds accumulator rows that are
+    // discarded): the cells behind the last row of each input plane, the planes of
+    // the unused upper 64 rows when CB = 64, and the gradient rows behind the tile.
     {
-        const uint32_t total16 = (kSlotsA * p.a_slot_bytes + p.slotsB * p.b_slot_bytes) / 16;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
-        for (uint32_t e = tid; e < total16; e += kThreads2) reinterpret_cast<uint4*>(smem_gen)[e] = zero4;
+        const int planes_alloc = (int)(p.a_slot_bytes / p.sbo_a);
+        const int planes_real = ncib * p.ncgpc;
+        const int cells = (int)(p.sbo_a / 16), written = p.rowsA * p.Wzq;
+        for (int s = 0; s < kSlotsA; ++s) {
+            for (int pl = warp; pl < planes_alloc; pl += kThreads2 / 32) {
+                uint4* plane = reinterpret_cast<uint4*>(smem_gen + (size_t)s * p.a_slot_bytes + (size_t)pl * p.sbo_a);
+                for (int c = (pl < planes_real ? written : 0) + lane; c < cells; c += 32) plane[c] = zero4;
+            }
+        }
+        const int tail0 = p.Ic * p.Wzq * 8, tail1 = p.KT * 8;      // in 16-byte units per chunk
+        unsigned char* bgen = smem_gen + (size_t)kSlotsA * p.a_slot_bytes;
+        for (int sc = warp; sc < p.slotsB * p.nchunks; sc += kThreads2 / 32) {
+            uint4* chunk = reinterpret_cast<uint4*>(bgen + (size_t)sc * p.b_chunk_bytes);
+            for (int c = tail0 + lane; c < tail1; c += 32) chunk[c] = zero4;
+        }
         fence_proxy_async_smem();
     }
     if (tid < p.ncls * kMaxUnits2) {
@@ -161,25 +176,30 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                     tma_load_4d(b_slot + c * p.b_chunk_bytes, &p.tmB[cls], &fullB[sb], co0 + 64 * c, 0, i0, n);
             }
         }
-    } else if (warp == 1 && lane == 0) {
+    } else if (warp == 1) {
         // ----------------------------------------------------------- MMA issuer
+        // The whole warp runs the loop so that the descriptor arithmetic stays in
+        // uniform registers; one elected lane issues each MMA and commit.
         const uint32_t idesc = make_idesc(p.BN);
         const uint32_t a_hi = desc_hi(p.sbo_a, 0);           // un-swizzled
         const uint32_t b_hi = desc_hi(1024, 2);              // 128-byte swizzle, 8 rows per atom
+        const bool leader = elect_one();
         int tb = 0;
         bool ok = true;
         for (int kt = kt_begin, ta = 0; kt < kt_end && ok; ++kt, ++ta) {
             const int sa = ta % kSlotsA;
-            if (!mbar_wait(&fullA[sa], (ta / kSlotsA) & 1, abort_flag)) {
-                flag_timeout(&abort_s, p.status, 0x200u + sa);
+            bool got = mbar_wait(&fullA[sa], (ta / kSlotsA) & 1, abort_flag);
+            if (!__all_sync(0xffffffffu, got)) {
+                if (leader) flag_timeout(&abort_s, p.status, 0x200u + sa);
                 ok = false;
                 break;
             }
             const uint32_t a_lo0 = desc_lo(a_base + sa * p.a_slot_bytes, 128);
             for (int cls = 0; cls < p.ncls; ++cls, ++tb) {
                 const int sb = tb % p.slotsB;
-                if (!mbar_wait(&fullB[sb], (tb / p.slotsB) & 1, abort_flag)) {
-                    flag_timeout(&abort_s, p.status, 0x280u + sb);
+                got = mbar_wait(&fullB[sb], (tb / p.slotsB) & 1, abort_flag);
+                if (!__all_sync(0xffffffffu, got)) {
+                    if (leader) flag_timeout(&abort_s, p.status, 0x280u + sb);
                     ok = false;
                     break;
                 }
@@ -190,18 +210,20 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                     uint32_t a_lo = a_lo0 + (aoff_tab[cls][u] >> 4);
                     uint32_t b_lo = b_lo0;
                     const uint32_t dcol = tmem_base + (uint32_t)u * p.BN;
-                    mma_bf16_words(dcol, a_lo, a_hi, b_lo, b_hi, idesc, first);
+                    if (leader) mma_bf16_words(dcol, a_lo, a_hi, b_lo, b_hi, idesc, first);
                     for (int kk = 1; kk < p.ksteps; ++kk) {
                         a_lo += 16;    // 16 cells x 16 bytes
                         b_lo += 128;   // 16 rows x 128 bytes
-                        mma_bf16_words(dcol, a_lo, a_hi, b_lo, b_hi, idesc, 1u);
+                        if (leader) mma_bf16_words(dcol, a_lo, a_hi, b_lo, b_hi, idesc, 1u);
                     }
                 }
-                mma_commit(&emptyB[sb]);
+                if (leader) mma_commit(&emptyB[sb]);
+                __syncwarp();
             }
-            if (ok) mma_commit(&emptyA[sa]);
+            if (ok && leader) mma_commit(&emptyA[sa]);
+            __syncwarp();
         }
-        if (ok) mma_commit(&done_bar);
+        if (ok && leader) mma_commit(&done_bar);
     }
     __syncwarp();
 
