@@ -88,44 +88,100 @@ __device__ __forceinline__ uint4 pack<__nv_bfloat16>(const float* f) {
 // One thread per output vector (n, p, q, 16 bytes of channels): k*k independent
 // 16-byte loads, element-wise fp32 sums, one 16-byte store. Adjacent threads
 // hold adjacent channel vectors, so every warp-wide access is contiguous.
-template <typename T, bool RELU>
+// Grid: x covers the (q, channel vector) pairs of one pooled row, y = p, z = n,
+// so that no 64-bit division is needed. K > 0: pooling factor known at compile
+// time, all loads of up to four rows issued before the first use; K = 0: any k.
+template <typename T, int K, bool RELU>
 __global__ void __launch_bounds__(256)
 compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W, int CV, int k,
-                  int Hp, int Wp, long long total) {
+                  int Hp, int Wp) {
     constexpr int VW = VecTraits<T>::VW;
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= total) return;
-    const int cv = (int)(idx % CV);
-    long long t = idx / CV;
-    const int q = (int)(t % Wp); t /= Wp;
-    const int p = (int)(t % Hp);
-    const long long n = t / Hp;
-    const int h0 = p * k, w0 = q * k;
-    const int h1 = min(h0 + k, H), w1 = min(w0 + k, W);
+    const unsigned item = blockIdx.x * 256u + threadIdx.x;
+    if (item >= (unsigned)Wp * (unsigned)CV) return;
+    const int q = (int)(item / (unsigned)CV);
+    const int cv = (int)(item - (unsigned)q * (unsigned)CV);
+    const int p = blockIdx.y;
+    const long long n = blockIdx.z;
+    const int kk = K > 0 ? K : k;
+    const int h0 = p * kk, w0 = q * kk;
+    const int h1 = min(h0 + kk, H), w1 = min(w0 + kk, W);
     float acc[VW];
 #pragma unroll
     for (int i = 0; i < VW; ++i) acc[i] = 0.f;
-    for (int h = h0; h < h1; ++h) {
-        float row[VW];
+    if (K > 0) {
+        constexpr int KR = K > 0 ? (K > 4 ? 2 : K) : 1;   // rows in flight at once
 #pragma unroll
-        for (int i = 0; i < VW; ++i) row[i] = 0.f;
-        const long long rbase = ((n * H + h) * (long long)W) * CV + cv;
-        for (int w = w0; w < w1; ++w) {
-            const long long off = (rbase + (long long)w * CV) * VW;
-            uint4 raw = load16<!RELU>(x + off);
-            float f[VW];
-            unpack<T, RELU>(raw, f);
-            if (RELU) *reinterpret_cast<uint4*>(y + off) = raw;
+        for (int hb = 0; hb < (K > 0 ? K : 1); hb += KR) {
+            uint4 raw[KR][K > 0 ? K : 1];
 #pragma unroll
-            for (int i = 0; i < VW; ++i) row[i] += f[i];
+            for (int dh = 0; dh < KR; ++dh)
+#pragma unroll
+                for (int dw = 0; dw < K; ++dw) {
+                    const int h = h0 + hb + dh, w = w0 + dw;
+                    raw[dh][dw] = make_uint4(0, 0, 0, 0);
+                    if (h < h1 && w < w1)
+                        raw[dh][dw] = load16<!RELU>(x + ((((n * H + h) * (long long)W + w) * CV + cv) * VW));
+                }
+#pragma unroll
+            for (int dh = 0; dh < KR; ++dh) {
+                float row[VW];
+#pragma unroll
+                for (int i = 0; i < VW; ++i) row[i] = 0.f;
+#pragma unroll
+                for (int dw = 0; dw < K; ++dw) {
+                    const int h = h0 + hb + dh, w = w0 + dw;
+                    float f[VW];
+                    unpack<T, RELU>(raw[dh][dw], f);
+                    if (RELU && h < h1 && w < w1)
+                        *reinterpret_cast<uint4*>(y + ((((n * H + h) * (long long)W + w) * CV + cv) * VW)) =
+                            raw[dh][dw];
+#pragma unroll
+                    for (int i = 0; i < VW; ++i) row[i] += f[i];
+                }
+#pragma unroll
+                for (int i = 0; i < VW; ++i) acc[i] += row[i];
+            }
         }
+    } else {
+        for (int h = h0; h < h1; ++h) {
+            float row[VW];
 #pragma unroll
-        for (int i = 0; i < VW; ++i) acc[i] += row[i];
+            for (int i = 0; i < VW; ++i) row[i] = 0.f;
+            const long long rbase = ((n * H + h) * (long long)W) * CV + cv;
+            for (int w = w0; w < w1; ++w) {
+                const long long off = (rbase + (long long)w * CV) * VW;
+                uint4 raw = load16<!RELU>(x + off);
+                float f[VW];
+                unpack<T, RELU>(raw, f);
+                if (RELU) *reinterpret_cast<uint4*>(y + off) = raw;
+#pragma unroll
+                for (int i = 0; i < VW; ++i) row[i] += f[i];
+            }
+#pragma unroll
+            for (int i = 0; i < VW; ++i) acc[i] += row[i];
+        }
     }
     const float inv = 1.0f / (float)((h1 - h0) * (w1 - w0));
 #pragma unroll
     for (int i = 0; i < VW; ++i) acc[i] *= inv;
-    *reinterpret_cast<uint4*>(z + idx * VW) = pack<T>(acc);
+    *reinterpret_cast<uint4*>(z + ((((n * Hp + p) * (long long)Wp + q) * CV + cv) * VW)) = pack<T>(acc);
+}
+
+template <typename T, bool RELU>
+ac_status launch_nhwc_vec(const T* x, T* z, T* y, long long N, int H, int W, int CV, int k, int Hp, int Wp,
+                          cudaStream_t st) {
+    const long long row_items = (long long)Wp * CV;
+    if (row_items >= (1ll << 31) || Hp > 65535 || N > 65535) return AC_ERR_UNSUPPORTED;
+    dim3 grid((unsigned)((row_items + 255) / 256), (unsigned)Hp, (unsigned)N);
+    switch (k) {
+        case 1: compress_nhwc_vec<T, 1, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
+        case 2: compress_nhwc_vec<T, 2, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
+        case 4: compress_nhwc_vec<T, 4, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
+        case 8: compress_nhwc_vec<T, 8, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
+        default: compress_nhwc_vec<T, 0, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
+    }
+    AC_CUDA_TRY(cudaGetLastError());
+    return AC_OK;
 }
 
 // ---- NCHW, W a multiple of the vector width and of k, k in {2,4,8} ---------
@@ -133,19 +189,20 @@ compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W
 // read consecutive 16-byte chunks of a row. Vertical sums over the k rows are
 // element-wise; the horizontal sum is a tree inside the vector, finished with
 // one warp shuffle when a block spans two lanes (fp32, k = 8).
-template <typename T, int K, bool RELU>
+template <typename T, int K, bool RELU, typename I>
 __global__ void __launch_bounds__(256)
 compress_nchw_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W, int Hp, int Wp,
                   long long total) {
     constexpr int VW = VecTraits<T>::VW;
     const int WV = W / VW;
-    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool active = idx < total;
-    if (!active) idx = total - 1;  // keep whole warps alive for the shuffle
-    const int wv = (int)(idx % WV);
-    long long t = idx / WV;
-    const int p = (int)(t % Hp);
-    const long long nc = t / Hp;
+    I idx = (I)blockIdx.x * 256u + threadIdx.x;     // I = unsigned when the item count fits 32 bits
+    const bool active = idx < (I)total;
+    if (!active) idx = (I)(total - 1);  // keep whole warps alive for the shuffle
+    const I t0 = idx / (I)WV;
+    const int wv = (int)(idx - t0 * (I)WV);
+    const I nci = t0 / (I)Hp;
+    const int p = (int)(t0 - nci * (I)Hp);
+    const long long nc = (long long)nci;
     const int h0 = p * K;
     const int h1 = min(h0 + K, H);
     float acc[VW];
@@ -224,6 +281,16 @@ compress_generic(const T* x, T* __restrict__ z, T* y, int C, int H, int W, int k
 
 inline unsigned blocks_for(long long total) { return (unsigned)((total + 255) / 256); }
 
+template <typename T, int K, bool RELU>
+void launch_nchw_vec(const Dims& d, const T* x, T* z, T* y, long long total, cudaStream_t st) {
+    const unsigned g = blocks_for(total);
+    if (total < (1ll << 32))
+        compress_nchw_vec<T, K, RELU, unsigned><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp, total);
+    else
+        compress_nchw_vec<T, K, RELU, unsigned long long><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp,
+                                                                              total);
+}
+
 template <typename T, bool RELU>
 ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, cudaStream_t st) {
     constexpr int VW = VecTraits<T>::VW;
@@ -233,27 +300,19 @@ ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, cudaStream_t st) {
     if (d.k == 1 && d.x_elems() % VW == 0) {
         // a copy (or a plain ReLU): treat the tensor as one row of 16-byte vectors
         const long long nv = d.x_elems() / VW;
-        if (nv < (1ll << 31)) {
-            compress_nhwc_vec<T, RELU><<<blocks_for(nv), 256, 0, st>>>(x, z, y, 1, (int)nv, 1, 1, 1,
-                                                                       (int)nv, nv);
-            AC_CUDA_TRY(cudaGetLastError());
-            return AC_OK;
-        }
+        if (nv < (1ll << 31))
+            return launch_nhwc_vec<T, RELU>(x, z, y, 1, 1, (int)nv, 1, 1, 1, (int)nv, st);
     }
     if (d.layout == AC_NHWC && d.Ci % VW == 0) {
-        const long long total = zt / VW;
-        compress_nhwc_vec<T, RELU><<<blocks_for(total), 256, 0, st>>>(x, z, y, d.H, d.W, d.Ci / VW,
-                                                                      d.k, d.Hp, d.Wp, total);
-    } else if (d.layout == AC_NCHW && pow2k && d.W % VW == 0 && d.W % d.k == 0 &&
-               (VW % d.k == 0 || d.k == 2 * VW)) {
+        const ac_status st_ = launch_nhwc_vec<T, RELU>(x, z, y, d.N, d.H, d.W, d.Ci / VW, d.k, d.Hp, d.Wp, st);
+        if (st_ != AC_ERR_UNSUPPORTED) return st_;
+    }
+    if (d.layout == AC_NCHW && pow2k && d.W % VW == 0 && d.W % d.k == 0 &&
+        (VW % d.k == 0 || d.k == 2 * VW)) {
         const long long total = (long long)d.N * d.Ci * d.Hp * (d.W / VW);
-        const unsigned g = blocks_for(total);
-        if (d.k == 2)
-            compress_nchw_vec<T, 2, RELU><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp, total);
-        else if (d.k == 4)
-            compress_nchw_vec<T, 4, RELU><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp, total);
-        else
-            compress_nchw_vec<T, 8, RELU><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp, total);
+        if (d.k == 2) launch_nchw_vec<T, 2, RELU>(d, x, z, y, total, st);
+        else if (d.k == 4) launch_nchw_vec<T, 4, RELU>(d, x, z, y, total, st);
+        else launch_nchw_vec<T, 8, RELU>(d, x, z, y, total, st);
     } else {
         compress_generic<T, RELU><<<blocks_for(zt), 256, 0, st>>>(
             x, z, y, d.Ci, d.H, d.W, d.k, d.Hp, d.Wp, d.layout == AC_NHWC, zt);
