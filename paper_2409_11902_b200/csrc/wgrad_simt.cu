@@ -151,10 +151,46 @@ splitk_reduce_kernel(const float* __restrict__ partials, int splits, long long e
     dw[i] = (s0 + s1) + (s2 + s3);
 }
 
+// Same sums, four consecutive elements per thread (elems % 4 == 0).
+__global__ void __launch_bounds__(256)
+splitk_reduce4_kernel(const float4* __restrict__ partials, int splits, long long elems4,
+                      float4* __restrict__ dw) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= elems4) return;
+    float4 s[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) s[a] = make_float4(0.f, 0.f, 0.f, 0.f);
+    int sp = 0;
+    for (; sp + 4 <= splits; sp += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) v[a] = __ldcs(partials + (long long)(sp + a) * elems4 + i);
+#pragma unroll
+        for (int a = 0; a < 4; ++a) { s[a].x += v[a].x; s[a].y += v[a].y; s[a].z += v[a].z; s[a].w += v[a].w; }
+    }
+    for (int a = 0; sp + a < splits; ++a) {
+        const float4 v = __ldcs(partials + (long long)(sp + a) * elems4 + i);
+        s[a].x += v.x; s[a].y += v.y; s[a].z += v.z; s[a].w += v.w;
+    }
+    float4 o;
+    o.x = (s[0].x + s[1].x) + (s[2].x + s[3].x);
+    o.y = (s[0].y + s[1].y) + (s[2].y + s[3].y);
+    o.z = (s[0].z + s[1].z) + (s[2].z + s[3].z);
+    o.w = (s[0].w + s[1].w) + (s[2].w + s[3].w);
+    dw[i] = o;
+}
+
 }  // namespace
 
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
                                cudaStream_t stream) {
+    if (elems % 4 == 0) {
+        const long long e4 = elems / 4;
+        splitk_reduce4_kernel<<<(unsigned)((e4 + 255) / 256), 256, 0, stream>>>(
+            reinterpret_cast<const float4*>(partials), splits, e4, reinterpret_cast<float4*>(dw));
+        AC_CUDA_TRY(cudaGetLastError());
+        return AC_OK;
+    }
     const unsigned grid = (unsigned)((elems + 255) / 256);
     splitk_reduce_kernel<<<grid, 256, 0, stream>>>(partials, splits, elems, dw);
     AC_CUDA_TRY(cudaGetLastError());

@@ -94,50 +94,106 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     unsigned char* smem_gen = tc2_smem + (smem_base - smem_u32(tc2_smem));
     const uint32_t a_base = smem_base, b_base = smem_base + kSlotsA * p.a_slot_bytes;
 
+    // ---------------------------------------------------------------- TMA producer
+    // Warp 0 issues every copy. The stream of copies is: for each K-tile, the Z halo
+    // tile (one copy per 8-channel plane, one plane per lane so that the planes of a
+    // tile go out as one warp instruction), then one gradient tile per class (one
+    // 64-channel chunk per lane). It is written as a resumable loop so that the first
+    // tiles, which need no free slot, are already in flight while the other warps do
+    // the set-up work below.
+    int pr_kt = kt_begin, pr_ta = 0, pr_cls = -1, pr_tb = 0;
+    auto produce = [&](bool may_wait) {
+        const int nplanes = ncib * p.ncgpc;
+        while (pr_kt < kt_end) {
+            const int n = pr_kt / p.bands, band = pr_kt - n * p.bands;
+            const int i0 = band * p.Ic;
+            if (pr_cls < 0) {
+                const int sa = pr_ta % kSlotsA;
+                if (pr_ta >= kSlotsA) {
+                    if (!may_wait) return;
+                    const bool got = mbar_wait(&emptyA[sa], ((pr_ta / kSlotsA) & 1) ^ 1, abort_flag);
+                    if (!__all_sync(0xffffffffu, got)) {
+                        if (lane == 0) flag_timeout(&abort_s, p.status, 0x100u + sa);
+                        return;
+                    }
+                }
+                if (lane == 0) mbar_arrive_expect_tx(&fullA[sa], (uint32_t)nplanes * p.a_box_bytes);
+                __syncwarp();
+                const uint32_t a_slot = a_base + sa * p.a_slot_bytes;
+                for (int pl = lane; pl < nplanes; pl += 32)
+                    tma_load_4d(a_slot + pl * p.sbo_a, &p.tmA, &fullA[sa], cib0 * p.CB + pl * 8, p.vmin,
+                                i0 + p.umin, n);
+                pr_cls = 0;
+            } else {
+                const int sb = pr_tb % p.slotsB;
+                if (pr_tb >= p.slotsB) {
+                    if (!may_wait) return;
+                    const bool got = mbar_wait(&emptyB[sb], ((pr_tb / p.slotsB) & 1) ^ 1, abort_flag);
+                    if (!__all_sync(0xffffffffu, got)) {
+                        if (lane == 0) flag_timeout(&abort_s, p.status, 0x180u + sb);
+                        return;
+                    }
+                }
+                if (lane == 0) mbar_arrive_expect_tx(&fullB[sb], (uint32_t)p.nchunks * p.b_box_bytes);
+                __syncwarp();
+                const uint32_t b_slot = b_base + sb * p.b_slot_bytes;
+                if (lane < p.nchunks)
+                    tma_load_4d(b_slot + lane * p.b_chunk_bytes, &p.tmB[pr_cls], &fullB[sb], co0 + 64 * lane, 0,
+                                i0, n);
+                ++pr_tb;
+                if (++pr_cls == p.ncls) { pr_cls = -1; ++pr_kt; ++pr_ta; }
+            }
+        }
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], 1); }
+            for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], 1); }
+            mbar_init(&done_bar, 1);
+            abort_s = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+        produce(false);   // fills every slot once; the copies only touch cells no one else writes
+    }
     // Everything the MMAs may read but no copy ever writes must be finite (it only
     // ever meets zeros of the other operand, or feeds accumulator rows that are
     // discarded): the cells behind the last row of each input plane, the planes of
     // the unused upper 64 rows when CB = 64, and the gradient rows behind the tile.
-    {
+    if (warp >= 1) {
+        constexpr int kZeroWarps = kThreads2 / 32 - 1;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         const int planes_alloc = (int)(p.a_slot_bytes / p.sbo_a);
         const int planes_real = ncib * p.ncgpc;
         const int cells = (int)(p.sbo_a / 16), written = p.rowsA * p.Wzq;
         for (int s = 0; s < kSlotsA; ++s) {
-            for (int pl = warp; pl < planes_alloc; pl += kThreads2 / 32) {
+            for (int pl = warp - 1; pl < planes_alloc; pl += kZeroWarps) {
                 uint4* plane = reinterpret_cast<uint4*>(smem_gen + (size_t)s * p.a_slot_bytes + (size_t)pl * p.sbo_a);
                 for (int c = (pl < planes_real ? written : 0) + lane; c < cells; c += 32) plane[c] = zero4;
             }
         }
         const int tail0 = p.Ic * p.Wzq * 8, tail1 = p.KT * 8;      // in 16-byte units per chunk
         unsigned char* bgen = smem_gen + (size_t)kSlotsA * p.a_slot_bytes;
-        for (int sc = warp; sc < p.slotsB * p.nchunks; sc += kThreads2 / 32) {
+        for (int sc = warp - 1; sc < p.slotsB * p.nchunks; sc += kZeroWarps) {
             uint4* chunk = reinterpret_cast<uint4*>(bgen + (size_t)sc * p.b_chunk_bytes);
             for (int c = tail0 + lane; c < tail1; c += 32) chunk[c] = zero4;
         }
         fence_proxy_async_smem();
-    }
-    if (tid < p.ncls * kMaxUnits2) {
-        const int cls = tid / kMaxUnits2, u = tid % kMaxUnits2;
-        uint32_t off = 0;
-        if (u < nunits) {
-            const int cl = u / ntap, t = u - cl * ntap;
-            const int tap = tap0 + t, r = tap / p.S, sx = tap - r * p.S;
-            const int a = cls / p.c_w, b = cls - a * p.c_w;
-            const int uu = floor_div_i(p.sh * a - p.ph + r, p.k) - p.umin;
-            const int vv = floor_div_i(p.sw * b - p.pw + sx, p.k) - p.vmin;
-            off = (uint32_t)(cl * p.ncgpc) * p.sbo_a + (uint32_t)(uu * p.Wzq + vv) * 16u;
+        const int t2 = tid - 32;
+        if (t2 < p.ncls * kMaxUnits2) {
+            const int cls = t2 / kMaxUnits2, u = t2 % kMaxUnits2;
+            uint32_t off = 0;
+            if (u < nunits) {
+                const int cl = u / ntap, t = u - cl * ntap;
+                const int tap = tap0 + t, r = tap / p.S, sx = tap - r * p.S;
+                const int a = cls / p.c_w, b = cls - a * p.c_w;
+                const int uu = floor_div_i(p.sh * a - p.ph + r, p.k) - p.umin;
+                const int vv = floor_div_i(p.sw * b - p.pw + sx, p.k) - p.vmin;
+                off = (uint32_t)(cl * p.ncgpc) * p.sbo_a + (uint32_t)(uu * p.Wzq + vv) * 16u;
+            }
+            aoff_tab[cls][u] = off;
         }
-        aoff_tab[cls][u] = off;
-    }
-    if (tid == 0) {
-        for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], 1); }
-        for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], 1); }
-        mbar_init(&done_bar, 1);
-        abort_s = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        prefetch_tmap(&p.tmA);
-        for (int c = 0; c < p.ncls; ++c) prefetch_tmap(&p.tmB[c]);
     }
     if (warp == 1) tmem_alloc(&tmem_base_s, p.tmem_cols);
     tc_fence_before();
@@ -145,37 +201,8 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
-    if (warp == 0 && lane == 0) {
-        // ---------------------------------------------------------- TMA producer
-        const int nplanes = ncib * p.ncgpc;
-        int tb = 0;
-        bool ok = true;
-        for (int kt = kt_begin, ta = 0; kt < kt_end && ok; ++kt, ++ta) {
-            const int sa = ta % kSlotsA;
-            if (ta >= kSlotsA && !mbar_wait(&emptyA[sa], ((ta / kSlotsA) & 1) ^ 1, abort_flag)) {
-                flag_timeout(&abort_s, p.status, 0x100u + sa);
-                break;
-            }
-            const int n = kt / p.bands, band = kt - n * p.bands;
-            const int i0 = band * p.Ic;
-            mbar_arrive_expect_tx(&fullA[sa], (uint32_t)nplanes * p.a_box_bytes);
-            const uint32_t a_slot = a_base + sa * p.a_slot_bytes;
-            for (int pl = 0; pl < nplanes; ++pl)
-                tma_load_4d(a_slot + pl * p.sbo_a, &p.tmA, &fullA[sa], cib0 * p.CB + pl * 8, p.vmin,
-                            i0 + p.umin, n);
-            for (int cls = 0; cls < p.ncls; ++cls, ++tb) {
-                const int sb = tb % p.slotsB;
-                if (tb >= p.slotsB && !mbar_wait(&emptyB[sb], ((tb / p.slotsB) & 1) ^ 1, abort_flag)) {
-                    flag_timeout(&abort_s, p.status, 0x180u + sb);
-                    ok = false;
-                    break;
-                }
-                mbar_arrive_expect_tx(&fullB[sb], (uint32_t)p.nchunks * p.b_box_bytes);
-                const uint32_t b_slot = b_base + sb * p.b_slot_bytes;
-                for (int c = 0; c < p.nchunks; ++c)
-                    tma_load_4d(b_slot + c * p.b_chunk_bytes, &p.tmB[cls], &fullB[sb], co0 + 64 * c, 0, i0, n);
-            }
-        }
+    if (warp == 0) {
+        produce(true);
     } else if (warp == 1) {
         // ----------------------------------------------------------- MMA issuer
         // The whole warp runs the loop so that the descriptor arithmetic stays in
@@ -237,21 +264,29 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             const int quarter = warp & 3;            // the TMEM lanes this warp may read
             const int m = quarter * 32 + lane;       // accumulator row
             float* dst = p.out + (long long)split * p.dw_elems;
-            int u = 0;
-            for (int cl = 0; cl < ncib; ++cl) {
-                const int ci = (cib0 + cl) * p.CB + m;
-                for (int t = 0; t < ntap; ++t, ++u) {
-                    const int tap = tap0 + t;
-                    for (int c0 = 0; c0 < p.BN; c0 += 32) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(u * p.BN + c0), r);
-                        if (m < p.CB) {
+            const long long cstride = (long long)RS * p.Ci;      // floats between output channels
+            const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            const int chunks_per_unit = p.BN / 32, nchunk = nunits * chunks_per_unit;
+            // 32 columns at a time, the next chunk's tcgen05.ld in flight while this one is stored
+            uint32_t buf[2][32];
+            tmem_ld32_issue(lane_base, buf[0]);
+            int u = 0, cu = 0;                        // unit and chunk-in-unit of chunk `ch`
+#pragma unroll 1
+            for (int ch = 0; ch < nchunk; ch += 2) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const long long o = ((long long)(co0 + c0 + j) * RS + tap) * p.Ci + ci;
-                                dst[o] = __uint_as_float(r[j]);
-                            }
+                for (int half = 0; half < 2; ++half) {
+                    if (ch + half < nchunk) {
+                        tmem_ld_wait();
+                        if (ch + half + 1 < nchunk)
+                            tmem_ld32_issue(lane_base + (uint32_t)((ch + half + 1) * 32), buf[half ^ 1]);
+                        const int cl = u / ntap, t = u - cl * ntap;
+                        if (m < p.CB) {
+                            float* q = dst + ((long long)(co0 + cu * 32) * RS + (tap0 + t)) * p.Ci +
+                                       (cib0 + cl) * p.CB + m;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) q[j * cstride] = __uint_as_float(buf[half][j]);
                         }
+                        if (++cu == chunks_per_unit) { cu = 0; ++u; }
                     }
                 }
             }
