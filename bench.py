@@ -108,6 +108,22 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(value: float, device) -> float:
+    """Slowest rank's time: the step time of a job whose replicas run side by side."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(world: int, flops_per_replica: int, ms: float) -> float:
+    """All replicas' work over the slowest replica's time (weak scaling)."""
+    return world * flops_per_replica / (ms * 1e-3) / 1e12
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -191,11 +207,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    total_ms = t0.elapsed_time(t1)
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(t0.elapsed_time(t1), dev)
 
     # Second live pass, same steps launched call by call with an event around every
     # C-ABI call: the per-kernel durations behind the roofline figures.
@@ -221,7 +233,7 @@ def run_ours(args):
     x_bytes = sum(d.N * d.C_in * d.H * d.W * elt for _, d in layers)
     z_bytes = sum(d.N * d.C_in * d.Hp * d.Wp * elt for _, d in layers)
     ms_per_step = total_ms / args.steps
-    value = world * sum(flops) / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tflops(world, sum(flops), ms_per_step)
     wg_tflops = sum(flops) / (sum(wgrad_ms) * 1e-3) / 1e12
     comp_gbs = sum(comp_bytes) / (sum(comp_ms) * 1e-3) / 1e9
     tensor_peak = peaks["bf16_tflops"]
@@ -251,12 +263,8 @@ def run_ours(args):
         e2e_step()
     t1.record(stream)
     torch.cuda.synchronize()
-    e2e_ms = t0.elapsed_time(t1) / n_e2e
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": world * sum(flops) / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1) / n_e2e, dev)
+    e2e = {"value": whole_job_tflops(world, sum(flops), e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms}
 
     if rank != 0:

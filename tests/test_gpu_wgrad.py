@@ -143,3 +143,44 @@ def test_host_step_matches_device_calls():
     ac.ac_conv2d_wgrad_compressed(d, z, dyd, dw, ws)
     torch.cuda.synchronize()
     assert torch.equal(z.cpu(), z_h) and torch.equal(dw.cpu(), dw_h)
+
+
+# Config 5: every distinct conv shape of ResNet-50 (bottleneck blocks, stride on the 3x3),
+# at a reduced batch; (C_in, C_out, H_in, R, stride, pad).
+RESNET50_SHAPES = [
+    (3, 64, 224, 7, 2, 3), (64, 64, 56, 1, 1, 0), (64, 64, 56, 3, 1, 1), (64, 256, 56, 1, 1, 0),
+    (256, 64, 56, 1, 1, 0), (256, 128, 56, 1, 1, 0), (128, 128, 56, 3, 2, 1), (128, 512, 28, 1, 1, 0),
+    (256, 512, 56, 1, 2, 0), (512, 128, 28, 1, 1, 0), (128, 128, 28, 3, 1, 1), (512, 256, 28, 1, 1, 0),
+    (256, 256, 28, 3, 2, 1), (256, 1024, 14, 1, 1, 0), (512, 1024, 28, 1, 2, 0), (1024, 256, 14, 1, 1, 0),
+    (256, 256, 14, 3, 1, 1), (1024, 512, 14, 1, 1, 0), (512, 512, 14, 3, 2, 1), (512, 2048, 7, 1, 1, 0),
+    (1024, 2048, 14, 1, 2, 0), (2048, 512, 7, 1, 1, 0), (512, 512, 7, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("Ci,Co,H,R,stride,pad", RESNET50_SHAPES)
+def test_resnet50_layer_shapes_sampled(Ci, Co, H, R, stride, pad):
+    N = 2 if H >= 56 else 8
+    err, _ = wgrad_error_sampled(D(N, Ci, Co, H, H, R, R, stride, pad, 2, "bf16", "nhwc"), n_samples=192)
+    assert err <= TOL_DW["bf16"], err
+
+
+def test_gradient_alignment_diagnostic():
+    """Section 5.2's cosine similarity between the compressed and the k = 1 weight
+    gradient, on synthetic data: 1 for k = 1, below 1 and decreasing with k, and the
+    GPU value equals the checker's."""
+    import oracle
+    from paper_2409_11902_b200 import synth
+    base = D(4, 64, 64, 16, 16, 3, 3, 1, 1, 1, "bf16", "nhwc")
+    x = synth.activation(3, (base.N, base.C_in, base.H, base.W), "bf16")
+    dy = synth.grad_output(3, (base.N, base.C_out, base.Ho, base.Wo), "bf16")
+    ref = run_wgrad(base, x, dy)
+    cos = {}
+    for k in (1, 2, 4):
+        d = dataclasses.replace(base, k=k)
+        z = synth.to_storage(oracle.pool(synth.to_f64(x), k), "bf16")
+        got = run_wgrad(d, z, dy)
+        cos[k] = oracle.cosine_similarity(got, ref)
+        want = oracle.wgrad_compressed(synth.to_f64(z), synth.to_f64(dy), 16, 16, 3, 3, (1, 1), (1, 1), k)
+        assert abs(cos[k] - oracle.cosine_similarity(want, ref)) < 1e-5
+    assert cos[1] == pytest.approx(1.0, abs=1e-9)
+    assert 0 < cos[4] < cos[2] < 1
