@@ -40,6 +40,10 @@ constexpr int kMaxClasses = 16;
 constexpr int kSlotsA = 2;
 constexpr int kMaxSlotsB = 8;
 constexpr uint32_t kSmemBudget2 = 220 * 1024;
+// Tap pairing for 64-channel layers (plan_pairs). Correct, but with one TMA copy per 8-channel
+// plane the extra tile copies cost more copy time than the saved MMAs: off until the tile
+// copies are cheap.
+constexpr bool kEnablePairs = false;
 
 struct Tc2Params {
     CUtensorMap tmA;                  // Z as (Ci, Wp, Hp, N)
@@ -55,6 +59,13 @@ struct Tc2Params {
     int slotsB;
     uint32_t a_slot_bytes, b_slot_bytes, b_chunk_bytes, sbo_a, a_box_bytes, b_box_bytes, tmem_cols;
     long long dw_elems;
+    // Paired mode (64 input channels): one accumulator tile holds TWO taps, rows 0-63
+    // tap A and rows 64-127 tap B, because the input tile is kept in up to three copies
+    // (8 planes each) shifted against each other; see plan_pairs().
+    int pair_mode, pu_count, ncopies;
+    int copy_du[3], copy_dv[3];                  // shift of copy g in Z rows / columns
+    signed char pu_tapA[kMaxUnits2], pu_tapB[kMaxUnits2];
+    unsigned int pu_off[kMaxClasses][kMaxUnits2];   // A start offset in bytes of (class, unit)
 };
 
 extern __shared__ __align__(1024) unsigned char tc2_smem[];
@@ -85,7 +96,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     const int ntap = min(p.taps_per_group, RS - tap0);
     const int cib0 = cibg * p.cibs_per_group;
     const int ncib = min(p.cibs_per_group, p.ncib_total - cib0);
-    const int nunits = ncib * ntap;
+    const int nunits = p.pair_mode ? p.pu_count : ncib * ntap;
     const int co0 = cob * p.BN;
     const int kt_begin = (int)((long long)p.ktiles * split / p.splits);
     const int kt_end = (int)((long long)p.ktiles * (split + 1) / p.splits);
@@ -103,7 +114,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     // the set-up work below.
     int pr_kt = kt_begin, pr_ta = 0, pr_cls = -1, pr_tb = 0;
     auto produce = [&](bool may_wait) {
-        const int nplanes = ncib * p.ncgpc;
+        const int nplanes = p.pair_mode ? 8 * p.ncopies : ncib * p.ncgpc;
         while (pr_kt < kt_end) {
             const int n = pr_kt / p.bands, band = pr_kt - n * p.bands;
             const int i0 = band * p.Ic;
@@ -120,9 +131,14 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 if (lane == 0) mbar_arrive_expect_tx(&fullA[sa], (uint32_t)nplanes * p.a_box_bytes);
                 __syncwarp();
                 const uint32_t a_slot = a_base + sa * p.a_slot_bytes;
-                for (int pl = lane; pl < nplanes; pl += 32)
-                    tma_load_4d(a_slot + pl * p.sbo_a, &p.tmA, &fullA[sa], cib0 * p.CB + pl * 8, p.vmin,
-                                i0 + p.umin, n);
+                for (int pl = lane; pl < nplanes; pl += 32) {
+                    // paired mode: plane pl belongs to copy pl / 8, the same 64 channels shifted
+                    const int g = p.pair_mode ? pl >> 3 : 0;
+                    const int ch = p.pair_mode ? (pl & 7) * 8 : pl * 8;
+                    const int dv = p.pair_mode ? p.copy_dv[g] : 0, du = p.pair_mode ? p.copy_du[g] : 0;
+                    tma_load_4d(a_slot + pl * p.sbo_a, &p.tmA, &fullA[sa], cib0 * p.CB + ch, p.vmin + dv,
+                                i0 + p.umin + du, n);
+                }
                 pr_cls = 0;
             } else {
                 const int sb = pr_tb % p.slotsB;
@@ -165,7 +181,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         constexpr int kZeroWarps = kThreads2 / 32 - 1;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         const int planes_alloc = (int)(p.a_slot_bytes / p.sbo_a);
-        const int planes_real = ncib * p.ncgpc;
+        const int planes_real = p.pair_mode ? 8 * p.ncopies : ncib * p.ncgpc;
         const int cells = (int)(p.sbo_a / 16), written = p.rowsA * p.Wzq;
         for (int s = 0; s < kSlotsA; ++s) {
             for (int pl = warp - 1; pl < planes_alloc; pl += kZeroWarps) {
@@ -184,7 +200,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         if (t2 < p.ncls * kMaxUnits2) {
             const int cls = t2 / kMaxUnits2, u = t2 % kMaxUnits2;
             uint32_t off = 0;
-            if (u < nunits) {
+            if (p.pair_mode) {
+                off = p.pu_off[cls][u];
+            } else if (u < nunits) {
                 const int cl = u / ntap, t = u - cl * ntap;
                 const int tap = tap0 + t, r = tap / p.S, sx = tap - r * p.S;
                 const int a = cls / p.c_w, b = cls - a * p.c_w;
@@ -279,10 +297,17 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                         tmem_ld_wait();
                         if (ch + half + 1 < nchunk)
                             tmem_ld32_issue(lane_base + (uint32_t)((ch + half + 1) * 32), buf[half ^ 1]);
-                        const int cl = u / ntap, t = u - cl * ntap;
-                        if (m < p.CB) {
-                            float* q = dst + ((long long)(co0 + cu * 32) * RS + (tap0 + t)) * p.Ci +
-                                       (cib0 + cl) * p.CB + m;
+                        int tap, ci;
+                        if (p.pair_mode) {
+                            tap = m < 64 ? p.pu_tapA[u] : p.pu_tapB[u];
+                            ci = cib0 * p.CB + (m & 63);
+                        } else {
+                            const int cl = u / ntap;
+                            tap = m < p.CB ? tap0 + (u - cl * ntap) : -1;
+                            ci = (cib0 + cl) * p.CB + m;
+                        }
+                        if (tap >= 0) {
+                            float* q = dst + ((long long)(co0 + cu * 32) * RS + tap) * p.Ci + ci;
 #pragma unroll
                             for (int j = 0; j < 32; ++j) q[j * cstride] = __uint_as_float(buf[half][j]);
                         }
@@ -305,6 +330,93 @@ struct Tc2Geom {
     double k_eff;
     bool ok;
 };
+
+// Pairing of taps for a layer with exactly 64 input channels. An MMA has M = 128 rows,
+// i.e. 16 planes of 8 channels read from consecutive plane slots; with 64 channels only
+// 8 planes are real. If the next 8 plane slots hold the SAME tile shifted by D cells,
+// rows 64-127 compute a second tap whose offset is D larger -- provided D is the same
+// for every output class. The tile is kept in up to three copies g = 0,1,2 with shifts
+// S0 = 0, S1 = D1, S2 = D1 + D2; a pair with difference D1 starts at copy 0, one with
+// difference D2 at copy 1, a tap without partner starts at copy 0 and wastes its upper
+// rows. Picks D1, D2 that pair the most taps. Returns false if nothing can be paired.
+struct PairPlan {
+    int count, ncopies;
+    int cu[3], cv[3];
+    int tapA[kMaxUnits2], tapB[kMaxUnits2], grp[kMaxUnits2];
+};
+
+bool plan_pairs(const Dims& d, int c_h, int c_w, int umin, int vmin, int uspan, int vspan, PairPlan* out) {
+    const int T = d.R * d.S, C = c_h * c_w;
+    if (T > 64) return false;
+    static thread_local int ou[kMaxClasses][64], ov[kMaxClasses][64];
+    for (int c = 0; c < C; ++c)
+        for (int t = 0; t < T; ++t) {
+            const int a = c / c_w, b = c % c_w, r = t / d.S, sx = t % d.S;
+            ou[c][t] = floor_div_i(d.sh * a - d.ph + r, d.k) - umin;
+            ov[c][t] = floor_div_i(d.sw * b - d.pw + sx, d.k) - vmin;
+        }
+    auto diff = [&](int t1, int t2, int* du, int* dv) {   // constant over classes?
+        *du = ou[0][t2] - ou[0][t1]; *dv = ov[0][t2] - ov[0][t1];
+        for (int c = 1; c < C; ++c)
+            if (ou[c][t2] - ou[c][t1] != *du || ov[c][t2] - ov[c][t1] != *dv) return false;
+        return true;
+    };
+    auto fits = [&](int t, int su, int sv) {              // tap t may start at a copy shifted by (su, sv)
+        for (int c = 0; c < C; ++c)
+            if (ou[c][t] - su < 0 || ou[c][t] - su > uspan || ov[c][t] - sv < 0 || ov[c][t] - sv > vspan)
+                return false;
+        return true;
+    };
+    int best_units = T;
+    PairPlan best{};
+    bool found = false;
+    for (int p1 = 0; p1 < T * T; ++p1) {
+        int d1u, d1v;
+        if (p1 / T == p1 % T || !diff(p1 / T, p1 % T, &d1u, &d1v)) continue;
+        for (int p2 = -1; p2 < T * T; ++p2) {
+            int d2u = 0, d2v = 0;
+            if (p2 >= 0 && (p2 / T == p2 % T || !diff(p2 / T, p2 % T, &d2u, &d2v))) continue;
+            bool used[64] = {};
+            PairPlan pp{};
+            for (int t1 = 0; t1 < T; ++t1) {                 // pairs at copy 0
+                if (used[t1]) continue;
+                for (int t2 = 0; t2 < T; ++t2) {
+                    int du, dv;
+                    if (t2 == t1 || used[t2] || !diff(t1, t2, &du, &dv) || du != d1u || dv != d1v) continue;
+                    if (pp.count >= kMaxUnits2) break;
+                    used[t1] = used[t2] = true;
+                    pp.tapA[pp.count] = t1; pp.tapB[pp.count] = t2; pp.grp[pp.count] = 0; ++pp.count;
+                    break;
+                }
+            }
+            bool any2 = false;
+            if (p2 >= 0) {
+                for (int t1 = 0; t1 < T; ++t1) {             // pairs at copy 1
+                    if (used[t1] || !fits(t1, d1u, d1v)) continue;
+                    for (int t2 = 0; t2 < T; ++t2) {
+                        int du, dv;
+                        if (t2 == t1 || used[t2] || !diff(t1, t2, &du, &dv) || du != d2u || dv != d2v) continue;
+                        if (pp.count >= kMaxUnits2) break;
+                        used[t1] = used[t2] = true; any2 = true;
+                        pp.tapA[pp.count] = t1; pp.tapB[pp.count] = t2; pp.grp[pp.count] = 1; ++pp.count;
+                        break;
+                    }
+                }
+            }
+            int units = pp.count;
+            for (int t = 0; t < T; ++t) units += used[t] ? 0 : 1;
+            if (units > kMaxUnits2 || units >= best_units) continue;
+            for (int t = 0; t < T; ++t)
+                if (!used[t]) { pp.tapA[pp.count] = t; pp.tapB[pp.count] = -1; pp.grp[pp.count] = 0; ++pp.count; }
+            pp.ncopies = any2 ? 3 : 2;
+            pp.cu[0] = 0; pp.cv[0] = 0; pp.cu[1] = d1u; pp.cv[1] = d1v;
+            pp.cu[2] = d1u + d2u; pp.cv[2] = d1v + d2v;
+            best = pp; best_units = units; found = true;
+        }
+    }
+    if (found) *out = best;
+    return found;
+}
 
 Tc2Geom make_geom2(const Dims& d) {
     Tc2Geom g{};
@@ -344,6 +456,21 @@ Tc2Geom make_geom2(const Dims& d) {
     p.taps_per_group = up.taps_per_group; p.ntapgroups = up.ntapgroups;
     p.cibs_per_group = up.cibs_per_group; p.ncibgroups = up.ncibgroups; p.groups = up.groups;
     p.tmem_cols = up.tmem_cols;
+    int planesA = up.planesA;
+    PairPlan pairs{};
+    p.pair_mode = 0;
+    if (kEnablePairs && d.Ci == 64 && plan_pairs(d, p.c_h, p.c_w, umin, vmin, g.uspan, g.vspan, &pairs) &&
+        pairs.count * up.BN <= 512) {
+        p.pair_mode = 1;
+        p.pu_count = pairs.count;
+        p.ncopies = pairs.ncopies;
+        for (int i = 0; i < 3; ++i) { p.copy_du[i] = pairs.cu[i]; p.copy_dv[i] = pairs.cv[i]; }
+        planesA = 8 * pairs.ncopies;
+        p.taps_per_group = d.R * d.S; p.ntapgroups = 1; p.cibs_per_group = 1; p.ncibgroups = 1;
+        p.groups = up.ncob;
+        p.tmem_cols = 32;
+        while (p.tmem_cols < (uint32_t)(pairs.count * up.BN)) p.tmem_cols *= 2;
+    }
 
     int best_Ic = 0, best_sb = 0;
     double best_eff = -1.0;
@@ -353,7 +480,7 @@ Tc2Geom make_geom2(const Dims& d) {
             const int KT = (Ic * p.Wzq + 15) / 16 * 16;
             const int NCa = (KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
             if ((uint32_t)NCa * 16 >= (1u << 18) || (uint32_t)KT * 128 >= (1u << 18)) break;
-            const uint32_t a_slot = ((uint32_t)up.planesA * NCa * 16 + 1023) / 1024 * 1024;
+            const uint32_t a_slot = ((uint32_t)planesA * NCa * 16 + 1023) / 1024 * 1024;
             const uint32_t b_slot = (uint32_t)p.nchunks * KT * 128;
             if (kSlotsA * a_slot + want * b_slot > kSmemBudget2) break;
             int sb = (int)((kSmemBudget2 - kSlotsA * a_slot) / b_slot);
@@ -373,7 +500,20 @@ Tc2Geom make_geom2(const Dims& d) {
     p.rowsA = p.Ic + g.uspan;
     const int NCa = (p.KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
     p.sbo_a = (uint32_t)NCa * 16;
-    p.a_slot_bytes = ((uint32_t)up.planesA * p.sbo_a + 1023) / 1024 * 1024;
+    p.a_slot_bytes = ((uint32_t)planesA * p.sbo_a + 1023) / 1024 * 1024;
+    if (p.pair_mode) {
+        for (int u = 0; u < pairs.count; ++u) {
+            p.pu_tapA[u] = (signed char)pairs.tapA[u];
+            p.pu_tapB[u] = (signed char)pairs.tapB[u];
+            const int gq = pairs.grp[u], t = pairs.tapA[u], r = t / d.S, sx = t % d.S;
+            for (int c = 0; c < p.ncls; ++c) {
+                const int a = c / p.c_w, b = c % p.c_w;
+                const int ouA = floor_div_i(d.sh * a - d.ph + r, d.k) - umin - pairs.cu[gq];
+                const int ovA = floor_div_i(d.sw * b - d.pw + sx, d.k) - vmin - pairs.cv[gq];
+                p.pu_off[c][u] = (uint32_t)(gq * 8) * p.sbo_a + (uint32_t)(ouA * p.Wzq + ovA) * 16u;
+            }
+        }
+    }
     p.b_chunk_bytes = (uint32_t)p.KT * 128;
     p.b_slot_bytes = (uint32_t)p.nchunks * p.b_chunk_bytes;
     p.a_box_bytes = 16u * p.Wzq * p.rowsA;
@@ -443,7 +583,7 @@ void tc2_plan_info(const Dims& d, ac_plan_info* info) {
     info->stages = g.p.slotsB;
     info->smem_bytes = (int32_t)g.smem_bytes;
     info->tmem_columns = (int32_t)g.p.tmem_cols;
-    info->units_per_cta = g.p.cibs_per_group * g.p.taps_per_group;
+    info->units_per_cta = g.p.pair_mode ? g.p.pu_count : g.p.cibs_per_group * g.p.taps_per_group;
     info->block_n = g.p.BN;
     info->a_cells = (int32_t)(g.p.sbo_a / 16);
     info->phases = g.p.ncls;
