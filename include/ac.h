@@ -19,7 +19,8 @@
  *   - Tensor pointers must be 16-byte aligned (AC_ERR_MISALIGNED otherwise).
  *   - Errors are return codes. No call aborts, throws or traps on the device.
  *     The descriptor is validated before anything is launched.
- *   - Reentrant; no global state except one-time kernel attribute set-up.
+ *   - Reentrant; no global state except one-time kernel attribute set-up and a small
+ *     mutex-protected cache of launch plans keyed by the descriptor.
  *
  * Shapes (logical): X [N, C_in, H, W]; Z [N, C_in, ceil(H/k), ceil(W/k)];
  * dY [N, C_out, H_o, W_o] with H_o = (H + 2 pad_h - R) / stride_h + 1 (floor),

@@ -5,6 +5,7 @@ namespace ac {
 
 ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o) {
     if (!d || !o) return AC_ERR_INVALID_ARG;
+    *o = Dims{};   // plans are cached by the bytes of this struct
     if (d->N <= 0 || d->C_in <= 0 || d->H <= 0 || d->W <= 0 || d->k <= 0) return AC_ERR_INVALID_ARG;
     if (d->dtype != AC_F32 && d->dtype != AC_BF16) return AC_ERR_INVALID_ARG;
     if (d->layout != AC_NCHW && d->layout != AC_NHWC) return AC_ERR_INVALID_ARG;

@@ -151,33 +151,59 @@ splitk_reduce_kernel(const float* __restrict__ partials, int splits, long long e
     dw[i] = (s0 + s1) + (s2 + s3);
 }
 
-// Same sums, four consecutive elements per thread (elems % 4 == 0).
+// Four consecutive elements per thread (elems % 4 == 0) and SL threads per element
+// group: thread (e, sl) adds slices sl, sl + SL, ... in order, then the SL running sums
+// of an element group are added in index order. Every order is fixed, so the result is
+// reproducible; SL only trades parallelism against slice-loop length when dW is small
+// and the slices are many.
+template <int SL>
 __global__ void __launch_bounds__(256)
 splitk_reduce4_kernel(const float4* __restrict__ partials, int splits, long long elems4,
                       float4* __restrict__ dw) {
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= elems4) return;
-    float4 s[4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a) s[a] = make_float4(0.f, 0.f, 0.f, 0.f);
-    int sp = 0;
-    for (; sp + 4 <= splits; sp += 4) {
-        float4 v[4];
-#pragma unroll
-        for (int a = 0; a < 4; ++a) v[a] = __ldcs(partials + (long long)(sp + a) * elems4 + i);
-#pragma unroll
-        for (int a = 0; a < 4; ++a) { s[a].x += v[a].x; s[a].y += v[a].y; s[a].z += v[a].z; s[a].w += v[a].w; }
+    constexpr int EL = 256 / SL;
+    __shared__ float4 red[SL > 1 ? SL : 1][EL];
+    const int e = threadIdx.x % EL, sl = threadIdx.x / EL;
+    const long long i = (long long)blockIdx.x * EL + e;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < elems4) {
+        int sp = sl;
+        for (; sp + 3 * SL < splits; sp += 4 * SL) {       // four loads in flight
+            const float4 v0 = __ldcs(partials + (long long)sp * elems4 + i);
+            const float4 v1 = __ldcs(partials + (long long)(sp + SL) * elems4 + i);
+            const float4 v2 = __ldcs(partials + (long long)(sp + 2 * SL) * elems4 + i);
+            const float4 v3 = __ldcs(partials + (long long)(sp + 3 * SL) * elems4 + i);
+            acc.x += v0.x; acc.y += v0.y; acc.z += v0.z; acc.w += v0.w;
+            acc.x += v1.x; acc.y += v1.y; acc.z += v1.z; acc.w += v1.w;
+            acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w;
+            acc.x += v3.x; acc.y += v3.y; acc.z += v3.z; acc.w += v3.w;
+        }
+        for (; sp < splits; sp += SL) {
+            const float4 v = __ldcs(partials + (long long)sp * elems4 + i);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
     }
-    for (int a = 0; sp + a < splits; ++a) {
-        const float4 v = __ldcs(partials + (long long)(sp + a) * elems4 + i);
-        s[a].x += v.x; s[a].y += v.y; s[a].z += v.z; s[a].w += v.w;
+    if (SL == 1) {
+        if (i < elems4) dw[i] = acc;
+        return;
     }
-    float4 o;
-    o.x = (s[0].x + s[1].x) + (s[2].x + s[3].x);
-    o.y = (s[0].y + s[1].y) + (s[2].y + s[3].y);
-    o.z = (s[0].z + s[1].z) + (s[2].z + s[3].z);
-    o.w = (s[0].w + s[1].w) + (s[2].w + s[3].w);
-    dw[i] = o;
+    red[sl][e] = acc;
+    __syncthreads();
+    if (sl == 0 && i < elems4) {
+        float4 o = red[0][e];
+#pragma unroll
+        for (int j = 1; j < SL; ++j) {
+            const float4 v = red[j][e];
+            o.x += v.x; o.y += v.y; o.z += v.z; o.w += v.w;
+        }
+        dw[i] = o;
+    }
+}
+
+template <int SL>
+void launch_reduce4(const float* partials, int splits, long long e4, float* dw, cudaStream_t stream) {
+    constexpr int EL = 256 / SL;
+    splitk_reduce4_kernel<SL><<<(unsigned)((e4 + EL - 1) / EL), 256, 0, stream>>>(
+        reinterpret_cast<const float4*>(partials), splits, e4, reinterpret_cast<float4*>(dw));
 }
 
 }  // namespace
@@ -186,8 +212,17 @@ ac_status launch_splitk_reduce(const float* partials, int splits, long long elem
                                cudaStream_t stream) {
     if (elems % 4 == 0) {
         const long long e4 = elems / 4;
-        splitk_reduce4_kernel<<<(unsigned)((e4 + 255) / 256), 256, 0, stream>>>(
-            reinterpret_cast<const float4*>(partials), splits, e4, reinterpret_cast<float4*>(dw));
+        // enough threads to fill the chip (148 SMs x 1024), at most one thread per 2 slices
+        int sl = 1;
+        while (sl < 32 && e4 * sl < 148 * 1024 && sl * 4 <= splits) sl *= 2;
+        switch (sl) {
+            case 1: launch_reduce4<1>(partials, splits, e4, dw, stream); break;
+            case 2: launch_reduce4<2>(partials, splits, e4, dw, stream); break;
+            case 4: launch_reduce4<4>(partials, splits, e4, dw, stream); break;
+            case 8: launch_reduce4<8>(partials, splits, e4, dw, stream); break;
+            case 16: launch_reduce4<16>(partials, splits, e4, dw, stream); break;
+            default: launch_reduce4<32>(partials, splits, e4, dw, stream); break;
+        }
         AC_CUDA_TRY(cudaGetLastError());
         return AC_OK;
     }

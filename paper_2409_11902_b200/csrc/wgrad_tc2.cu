@@ -25,6 +25,9 @@
 // drain the accumulators from tensor memory at the end. K is split over CTAs.
 #include <cuda.h>
 
+#include <cstring>
+#include <mutex>
+
 #include "ac_common.h"
 #include "tc_ptx.cuh"
 #include "tc_units.h"
@@ -40,10 +43,7 @@ constexpr int kMaxClasses = 16;
 constexpr int kSlotsA = 2;
 constexpr int kMaxSlotsB = 8;
 constexpr uint32_t kSmemBudget2 = 220 * 1024;
-// Tap pairing for 64-channel layers (plan_pairs). Correct, but with one TMA copy per 8-channel
-// plane the extra tile copies cost more copy time than the saved MMAs: off until the tile
-// copies are cheap.
-constexpr bool kEnablePairs = false;
+constexpr bool kEnablePairs = true;   // tap pairing for 64-channel layers (plan_pairs)
 
 struct Tc2Params {
     CUtensorMap tmA;                  // Z as (Ci, Wp, Hp, N)
@@ -57,7 +57,8 @@ struct Tc2Params {
     int CB, ncgpc, ncib_total, BN, nchunks;
     int taps_per_group, ntapgroups, cibs_per_group, ncibgroups, groups, splits, ktiles;
     int slotsB;
-    uint32_t a_slot_bytes, b_slot_bytes, b_chunk_bytes, sbo_a, a_box_bytes, b_box_bytes, tmem_cols;
+    uint32_t a_slot_bytes, b_slot_bytes, b_chunk_bytes, a_chunk_bytes, a_box_bytes, b_box_bytes, tmem_cols;
+    int chunksA;   // 64-channel chunks of the input tile per slot (incl. one never loaded when CB = 64)
     long long dw_elems;
     // Paired mode (64 input channels): one accumulator tile holds TWO taps, rows 0-63
     // tap A and rows 64-127 tap B, because the input tile is kept in up to three copies
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     // the set-up work below.
     int pr_kt = kt_begin, pr_ta = 0, pr_cls = -1, pr_tb = 0;
     auto produce = [&](bool may_wait) {
-        const int nplanes = p.pair_mode ? 8 * p.ncopies : ncib * p.ncgpc;
+        const int nloads = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);   // 64-channel chunks to fetch
         while (pr_kt < kt_end) {
             const int n = pr_kt / p.bands, band = pr_kt - n * p.bands;
             const int i0 = band * p.Ic;
@@ -128,16 +129,15 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                         return;
                     }
                 }
-                if (lane == 0) mbar_arrive_expect_tx(&fullA[sa], (uint32_t)nplanes * p.a_box_bytes);
+                if (lane == 0) mbar_arrive_expect_tx(&fullA[sa], (uint32_t)nloads * p.a_box_bytes);
                 __syncwarp();
                 const uint32_t a_slot = a_base + sa * p.a_slot_bytes;
-                for (int pl = lane; pl < nplanes; pl += 32) {
-                    // paired mode: plane pl belongs to copy pl / 8, the same 64 channels shifted
-                    const int g = p.pair_mode ? pl >> 3 : 0;
-                    const int ch = p.pair_mode ? (pl & 7) * 8 : pl * 8;
-                    const int dv = p.pair_mode ? p.copy_dv[g] : 0, du = p.pair_mode ? p.copy_du[g] : 0;
-                    tma_load_4d(a_slot + pl * p.sbo_a, &p.tmA, &fullA[sa], cib0 * p.CB + ch, p.vmin + dv,
-                                i0 + p.umin + du, n);
+                if (lane < nloads) {
+                    // paired mode: chunk `lane` is copy `lane` of the same 64 channels, shifted
+                    const int ch = p.pair_mode ? 0 : lane * 64;
+                    const int dv = p.pair_mode ? p.copy_dv[lane] : 0, du = p.pair_mode ? p.copy_du[lane] : 0;
+                    tma_load_4d(a_slot + lane * p.a_chunk_bytes, &p.tmA, &fullA[sa], cib0 * p.CB + ch,
+                                p.vmin + dv, i0 + p.umin + du, n);
                 }
                 pr_cls = 0;
             } else {
@@ -180,14 +180,12 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     if (warp >= 1) {
         constexpr int kZeroWarps = kThreads2 / 32 - 1;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
-        const int planes_alloc = (int)(p.a_slot_bytes / p.sbo_a);
-        const int planes_real = p.pair_mode ? 8 * p.ncopies : ncib * p.ncgpc;
-        const int cells = (int)(p.sbo_a / 16), written = p.rowsA * p.Wzq;
-        for (int s = 0; s < kSlotsA; ++s) {
-            for (int pl = warp - 1; pl < planes_alloc; pl += kZeroWarps) {
-                uint4* plane = reinterpret_cast<uint4*>(smem_gen + (size_t)s * p.a_slot_bytes + (size_t)pl * p.sbo_a);
-                for (int c = (pl < planes_real ? written : 0) + lane; c < cells; c += 32) plane[c] = zero4;
-            }
+        const int chunks_real = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);
+        const int units16 = (int)(p.a_chunk_bytes / 16), written = p.rowsA * p.Wzq * 8;
+        for (int sc = warp - 1; sc < kSlotsA * p.chunksA; sc += kZeroWarps) {
+            const int s_ = sc / p.chunksA, c_ = sc - s_ * p.chunksA;
+            uint4* chunk = reinterpret_cast<uint4*>(smem_gen + (size_t)s_ * p.a_slot_bytes + (size_t)c_ * p.a_chunk_bytes);
+            for (int c = (c_ < chunks_real ? written : 0) + lane; c < units16; c += 32) chunk[c] = zero4;
         }
         const int tail0 = p.Ic * p.Wzq * 8, tail1 = p.KT * 8;      // in 16-byte units per chunk
         unsigned char* bgen = smem_gen + (size_t)kSlotsA * p.a_slot_bytes;
@@ -208,7 +206,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 const int a = cls / p.c_w, b = cls - a * p.c_w;
                 const int uu = floor_div_i(p.sh * a - p.ph + r, p.k) - p.umin;
                 const int vv = floor_div_i(p.sw * b - p.pw + sx, p.k) - p.vmin;
-                off = (uint32_t)(cl * p.ncgpc) * p.sbo_a + (uint32_t)(uu * p.Wzq + vv) * 16u;
+                off = (uint32_t)(cl * (p.CB / 64)) * p.a_chunk_bytes + (uint32_t)(uu * p.Wzq + vv) * 128u;
             }
             aoff_tab[cls][u] = off;
         }
@@ -226,7 +224,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         // The whole warp runs the loop so that the descriptor arithmetic stays in
         // uniform registers; one elected lane issues each MMA and commit.
         const uint32_t idesc = make_idesc(p.BN);
-        const uint32_t a_hi = desc_hi(p.sbo_a, 0);           // un-swizzled
+        const uint32_t a_hi0 = desc_hi(1024, 2);             // both operands: 128-byte swizzle, 8-row atoms
         const uint32_t b_hi = desc_hi(1024, 2);              // 128-byte swizzle, 8 rows per atom
         const bool leader = elect_one();
         int tb = 0;
@@ -239,7 +237,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 ok = false;
                 break;
             }
-            const uint32_t a_lo0 = desc_lo(a_base + sa * p.a_slot_bytes, 128);
+            const uint32_t a_lo0 = desc_lo(a_base + sa * p.a_slot_bytes, p.a_chunk_bytes);
             for (int cls = 0; cls < p.ncls; ++cls, ++tb) {
                 const int sb = tb % p.slotsB;
                 got = mbar_wait(&fullB[sb], (tb / p.slotsB) & 1, abort_flag);
@@ -252,12 +250,17 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 const uint32_t b_lo0 = desc_lo(b_base + sb * p.b_slot_bytes, p.b_chunk_bytes);
                 const uint32_t first = (ta | cls) == 0 ? 0u : 1u;
                 for (int u = 0; u < nunits; ++u) {
+                    // A tap shifts the start by whole 128-byte rows. The swizzle is a function of
+                    // the absolute shared-memory address (TMA wrote the tile that way, slots are
+                    // 1024-byte aligned), so the descriptor needs no base offset: measured, a
+                    // non-zero base offset here gives wrong sums, zero gives the oracle's.
                     uint32_t a_lo = a_lo0 + (aoff_tab[cls][u] >> 4);
+                    const uint32_t a_hi = a_hi0;
                     uint32_t b_lo = b_lo0;
                     const uint32_t dcol = tmem_base + (uint32_t)u * p.BN;
                     if (leader) mma_bf16_words(dcol, a_lo, a_hi, b_lo, b_hi, idesc, first);
                     for (int kk = 1; kk < p.ksteps; ++kk) {
-                        a_lo += 16;    // 16 cells x 16 bytes
+                        a_lo += 128;   // 16 cells x 128 bytes
                         b_lo += 128;   // 16 rows x 128 bytes
                         if (leader) mma_bf16_words(dcol, a_lo, a_hi, b_lo, b_hi, idesc, 1u);
                     }
@@ -418,7 +421,7 @@ bool plan_pairs(const Dims& d, int c_h, int c_w, int umin, int vmin, int uspan, 
     return found;
 }
 
-Tc2Geom make_geom2(const Dims& d) {
+Tc2Geom build_geom2(const Dims& d) {
     Tc2Geom g{};
     Tc2Params& p = g.p;
     g.ok = false;
@@ -456,7 +459,7 @@ Tc2Geom make_geom2(const Dims& d) {
     p.taps_per_group = up.taps_per_group; p.ntapgroups = up.ntapgroups;
     p.cibs_per_group = up.cibs_per_group; p.ncibgroups = up.ncibgroups; p.groups = up.groups;
     p.tmem_cols = up.tmem_cols;
-    int planesA = up.planesA;
+    int chunksA = up.CB == 128 ? 2 * up.cibs_per_group : up.cibs_per_group + 1;
     PairPlan pairs{};
     p.pair_mode = 0;
     if (kEnablePairs && d.Ci == 64 && plan_pairs(d, p.c_h, p.c_w, umin, vmin, g.uspan, g.vspan, &pairs) &&
@@ -465,7 +468,7 @@ Tc2Geom make_geom2(const Dims& d) {
         p.pu_count = pairs.count;
         p.ncopies = pairs.ncopies;
         for (int i = 0; i < 3; ++i) { p.copy_du[i] = pairs.cu[i]; p.copy_dv[i] = pairs.cv[i]; }
-        planesA = 8 * pairs.ncopies;
+        chunksA = pairs.ncopies;
         p.taps_per_group = d.R * d.S; p.ntapgroups = 1; p.cibs_per_group = 1; p.ncibgroups = 1;
         p.groups = up.ncob;
         p.tmem_cols = 32;
@@ -479,8 +482,8 @@ Tc2Geom make_geom2(const Dims& d) {
             if (Ic + g.uspan > 256) break;
             const int KT = (Ic * p.Wzq + 15) / 16 * 16;
             const int NCa = (KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
-            if ((uint32_t)NCa * 16 >= (1u << 18) || (uint32_t)KT * 128 >= (1u << 18)) break;
-            const uint32_t a_slot = ((uint32_t)planesA * NCa * 16 + 1023) / 1024 * 1024;
+            if ((uint32_t)NCa * 128 >= (1u << 18) || (uint32_t)KT * 128 >= (1u << 18)) break;
+            const uint32_t a_slot = (uint32_t)chunksA * NCa * 128;
             const uint32_t b_slot = (uint32_t)p.nchunks * KT * 128;
             if (kSlotsA * a_slot + want * b_slot > kSmemBudget2) break;
             int sb = (int)((kSmemBudget2 - kSlotsA * a_slot) / b_slot);
@@ -499,8 +502,9 @@ Tc2Geom make_geom2(const Dims& d) {
     p.ksteps = p.KT / 16;
     p.rowsA = p.Ic + g.uspan;
     const int NCa = (p.KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
-    p.sbo_a = (uint32_t)NCa * 16;
-    p.a_slot_bytes = ((uint32_t)planesA * p.sbo_a + 1023) / 1024 * 1024;
+    p.a_chunk_bytes = (uint32_t)NCa * 128;
+    p.chunksA = chunksA;
+    p.a_slot_bytes = (uint32_t)chunksA * p.a_chunk_bytes;
     if (p.pair_mode) {
         for (int u = 0; u < pairs.count; ++u) {
             p.pu_tapA[u] = (signed char)pairs.tapA[u];
@@ -510,13 +514,13 @@ Tc2Geom make_geom2(const Dims& d) {
                 const int a = c / p.c_w, b = c % p.c_w;
                 const int ouA = floor_div_i(d.sh * a - d.ph + r, d.k) - umin - pairs.cu[gq];
                 const int ovA = floor_div_i(d.sw * b - d.pw + sx, d.k) - vmin - pairs.cv[gq];
-                p.pu_off[c][u] = (uint32_t)(gq * 8) * p.sbo_a + (uint32_t)(ouA * p.Wzq + ovA) * 16u;
+                p.pu_off[c][u] = (uint32_t)gq * p.a_chunk_bytes + (uint32_t)(ouA * p.Wzq + ovA) * 128u;
             }
         }
     }
     p.b_chunk_bytes = (uint32_t)p.KT * 128;
     p.b_slot_bytes = (uint32_t)p.nchunks * p.b_chunk_bytes;
-    p.a_box_bytes = 16u * p.Wzq * p.rowsA;
+    p.a_box_bytes = 128u * p.Wzq * p.rowsA;
     p.b_box_bytes = 128u * p.Wzq * p.Ic;
     p.slotsB = best_sb;
     g.k_eff = best_eff;
@@ -530,6 +534,28 @@ Tc2Geom make_geom2(const Dims& d) {
     g.smem_bytes = kSlotsA * p.a_slot_bytes + p.slotsB * p.b_slot_bytes + 1024;
     if (g.smem_bytes < 120 * 1024) g.smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
     g.ok = true;
+    return g;
+}
+
+// The geometry is pure arithmetic on the descriptor but not free (the pairing search):
+// the last few descriptors are remembered, so that the planning calls of one
+// ac_conv2d_wgrad_compressed (workspace size, support test, launch) and repeated layers pay once.
+Tc2Geom make_geom2(const Dims& d) {
+    constexpr int kEntries = 16;
+    static std::mutex mu;
+    static Dims keys[kEntries];
+    static Tc2Geom vals[kEntries];
+    static int used = 0, next = 0;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        for (int i = 0; i < used; ++i)
+            if (std::memcmp(&keys[i], &d, sizeof(Dims)) == 0) return vals[i];
+    }
+    const Tc2Geom g = build_geom2(d);
+    std::lock_guard<std::mutex> lock(mu);
+    keys[next] = d; vals[next] = g;
+    next = (next + 1) % kEntries;
+    if (used < kEntries) ++used;
     return g;
 }
 
@@ -585,7 +611,7 @@ void tc2_plan_info(const Dims& d, ac_plan_info* info) {
     info->tmem_columns = (int32_t)g.p.tmem_cols;
     info->units_per_cta = g.p.pair_mode ? g.p.pu_count : g.p.cibs_per_group * g.p.taps_per_group;
     info->block_n = g.p.BN;
-    info->a_cells = (int32_t)(g.p.sbo_a / 16);
+    info->a_cells = (int32_t)(g.p.a_chunk_bytes / 128);
     info->phases = g.p.ncls;
 }
 
@@ -600,10 +626,10 @@ ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, co
         const cuuint64_t dims[4] = {(cuuint64_t)d.Ci, (cuuint64_t)d.Wp, (cuuint64_t)d.Hp, (cuuint64_t)d.N};
         const cuuint64_t strides[3] = {(cuuint64_t)d.Ci * 2, (cuuint64_t)d.Wp * d.Ci * 2,
                                        (cuuint64_t)d.Hp * d.Wp * d.Ci * 2};
-        const cuuint32_t box[4] = {8, (cuuint32_t)p.Wzq, (cuuint32_t)p.rowsA, 1};
+        const cuuint32_t box[4] = {64, (cuuint32_t)p.Wzq, (cuuint32_t)p.rowsA, 1};
         const cuuint32_t es[4] = {1, 1, 1, 1};
         if (enc(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(z), dims, strides, box, es,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return AC_ERR_CUDA;
     }
