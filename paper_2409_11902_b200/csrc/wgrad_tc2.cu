@@ -54,6 +54,7 @@ struct Tc2Params {
     int c_h, c_w, ncls;
     int umin, vmin;
     int Wzq, Ic, bands, KT, ksteps, rowsA;
+    int NB, rowsB;   // images per K-tile (> 1 only when a tile is a whole class image) and dY rows per image
     int CB, ncgpc, ncib_total, BN, nchunks;
     int taps_per_group, ntapgroups, cibs_per_group, ncibgroups, groups, splits, ktiles;
     int slotsB;
@@ -117,8 +118,8 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     auto produce = [&](bool may_wait) {
         const int nloads = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);   // 64-channel chunks to fetch
         while (pr_kt < kt_end) {
-            const int n = pr_kt / p.bands, band = pr_kt - n * p.bands;
-            const int i0 = band * p.Ic;
+            const int n = p.NB > 1 ? pr_kt * p.NB : pr_kt / p.bands;
+            const int i0 = p.NB > 1 ? 0 : (pr_kt - n * p.bands) * p.Ic;
             if (pr_cls < 0) {
                 const int sa = pr_ta % kSlotsA;
                 if (pr_ta >= kSlotsA) {
@@ -181,13 +182,13 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         constexpr int kZeroWarps = kThreads2 / 32 - 1;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         const int chunks_real = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);
-        const int units16 = (int)(p.a_chunk_bytes / 16), written = p.rowsA * p.Wzq * 8;
+        const int units16 = (int)(p.a_chunk_bytes / 16), written = p.NB * p.rowsA * p.Wzq * 8;
         for (int sc = warp - 1; sc < kSlotsA * p.chunksA; sc += kZeroWarps) {
             const int s_ = sc / p.chunksA, c_ = sc - s_ * p.chunksA;
             uint4* chunk = reinterpret_cast<uint4*>(smem_gen + (size_t)s_ * p.a_slot_bytes + (size_t)c_ * p.a_chunk_bytes);
             for (int c = (c_ < chunks_real ? written : 0) + lane; c < units16; c += 32) chunk[c] = zero4;
         }
-        const int tail0 = p.Ic * p.Wzq * 8, tail1 = p.KT * 8;      // in 16-byte units per chunk
+        const int tail0 = p.NB * p.rowsB * p.Wzq * 8, tail1 = p.KT * 8;      // in 16-byte units per chunk
         unsigned char* bgen = smem_gen + (size_t)kSlotsA * p.a_slot_bytes;
         for (int sc = warp - 1; sc < p.slotsB * p.nchunks; sc += kZeroWarps) {
             uint4* chunk = reinterpret_cast<uint4*>(bgen + (size_t)sc * p.b_chunk_bytes);
@@ -475,32 +476,48 @@ Tc2Geom build_geom2(const Dims& d) {
         while (p.tmem_cols < (uint32_t)(pairs.count * up.BN)) p.tmem_cols *= 2;
     }
 
-    int best_Ic = 0, best_sb = 0;
-    double best_eff = -1.0;
+    // K-tile shape: Ic class rows of one image, or NB whole class images (then the gradient
+    // tile keeps the input tile's row count per image so that both stay on one flat pitch;
+    // the surplus rows are beyond the class's extent and arrive as zeros). Chosen by a cost
+    // model per image: a class tile costs max(MMA time, issue time + fixed turn-around),
+    // measured at about 80 cycles per MMA issued and 400 cycles per tile.
+    const int U = p.pair_mode ? pairs.count : up.units;
+    const double mma_clk = up.BN >= 128 ? up.BN / 2.0 : 48.0;   // N = 64 is shared-memory-read bound
+    int best_Ic = 0, best_sb = 0, best_NB = 1;
+    double best_cost = 1e30, best_eff = 0.0;
     for (int want = 3; want >= 2 && best_Ic == 0; --want) {
         for (int Ic = 1; Ic <= I; ++Ic) {
             if (Ic + g.uspan > 256) break;
-            const int KT = (Ic * p.Wzq + 15) / 16 * 16;
-            const int NCa = (KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
-            if ((uint32_t)NCa * 128 >= (1u << 18) || (uint32_t)KT * 128 >= (1u << 18)) break;
-            const uint32_t a_slot = (uint32_t)chunksA * NCa * 128;
-            const uint32_t b_slot = (uint32_t)p.nchunks * KT * 128;
-            if (kSlotsA * a_slot + want * b_slot > kSmemBudget2) break;
-            int sb = (int)((kSmemBudget2 - kSlotsA * a_slot) / b_slot);
-            if (sb > kMaxSlotsB) sb = kMaxSlotsB;
-            const int bands = (I + Ic - 1) / Ic;
-            const double eff = (double)d.Ho * d.Wo / ((double)bands * p.ncls * KT);
-            if (eff > best_eff + 1e-9 || (eff > best_eff - 1e-9 && Ic > best_Ic)) {
-                best_eff = eff; best_Ic = Ic; best_sb = sb;
+            for (int NB = 1; NB <= (Ic == I ? 16 : 1) && NB <= d.N; ++NB) {
+                const int rowsA = Ic + g.uspan;
+                const int KT = ((NB == 1 ? Ic : NB * rowsA) * p.Wzq + 15) / 16 * 16;
+                const int NCa = (KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
+                if ((uint32_t)NCa * 128 >= (1u << 18) || (uint32_t)KT * 128 >= (1u << 18)) break;
+                const uint32_t a_slot = (uint32_t)chunksA * NCa * 128;
+                const uint32_t b_slot = (uint32_t)p.nchunks * KT * 128;
+                if (kSlotsA * a_slot + want * b_slot > kSmemBudget2) break;
+                int sb = (int)((kSmemBudget2 - kSlotsA * a_slot) / b_slot);
+                if (sb > kMaxSlotsB) sb = kMaxSlotsB;
+                const int bands = (I + Ic - 1) / Ic;
+                const double tiles_per_image = NB == 1 ? (double)bands : 1.0 / NB;
+                const double mmas = (double)U * (KT / 16);
+                const double tile = mmas * mma_clk > 400.0 + 80.0 * mmas ? mmas * mma_clk : 400.0 + 80.0 * mmas;
+                const double cost = tiles_per_image * p.ncls * tile;
+                if (cost < best_cost * (1.0 - 1e-9)) {
+                    best_cost = cost; best_Ic = Ic; best_sb = sb; best_NB = NB;
+                    best_eff = (double)d.Ho * d.Wo / (tiles_per_image * p.ncls * KT);
+                }
             }
         }
     }
     if (best_Ic == 0) return g;
     p.Ic = best_Ic;
+    p.NB = best_NB;
     p.bands = (I + p.Ic - 1) / p.Ic;
-    p.KT = (p.Ic * p.Wzq + 15) / 16 * 16;
-    p.ksteps = p.KT / 16;
     p.rowsA = p.Ic + g.uspan;
+    p.rowsB = p.NB > 1 ? p.rowsA : p.Ic;
+    p.KT = ((p.NB == 1 ? p.Ic : p.NB * p.rowsA) * p.Wzq + 15) / 16 * 16;
+    p.ksteps = p.KT / 16;
     const int NCa = (p.KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
     p.a_chunk_bytes = (uint32_t)NCa * 128;
     p.chunksA = chunksA;
@@ -520,11 +537,11 @@ Tc2Geom build_geom2(const Dims& d) {
     }
     p.b_chunk_bytes = (uint32_t)p.KT * 128;
     p.b_slot_bytes = (uint32_t)p.nchunks * p.b_chunk_bytes;
-    p.a_box_bytes = 128u * p.Wzq * p.rowsA;
-    p.b_box_bytes = 128u * p.Wzq * p.Ic;
+    p.a_box_bytes = 128u * p.Wzq * p.rowsA * p.NB;
+    p.b_box_bytes = 128u * p.Wzq * p.rowsB * p.NB;
     p.slotsB = best_sb;
     g.k_eff = best_eff;
-    const long long ktiles = (long long)d.N * p.bands;
+    const long long ktiles = p.NB > 1 ? (d.N + p.NB - 1) / p.NB : (long long)d.N * p.bands;
     if (ktiles >= (1ll << 30)) return g;
     p.ktiles = (int)ktiles;
     int splits = kNumSMs / p.groups;
@@ -626,7 +643,7 @@ ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, co
         const cuuint64_t dims[4] = {(cuuint64_t)d.Ci, (cuuint64_t)d.Wp, (cuuint64_t)d.Hp, (cuuint64_t)d.N};
         const cuuint64_t strides[3] = {(cuuint64_t)d.Ci * 2, (cuuint64_t)d.Wp * d.Ci * 2,
                                        (cuuint64_t)d.Hp * d.Wp * d.Ci * 2};
-        const cuuint32_t box[4] = {64, (cuuint32_t)p.Wzq, (cuuint32_t)p.rowsA, 1};
+        const cuuint32_t box[4] = {64, (cuuint32_t)p.Wzq, (cuuint32_t)p.rowsA, (cuuint32_t)p.NB};
         const cuuint32_t es[4] = {1, 1, 1, 1};
         if (enc(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(z), dims, strides, box, es,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -640,7 +657,7 @@ ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, co
             const cuuint64_t dims[4] = {(cuuint64_t)d.Co, (cuuint64_t)Jb, (cuuint64_t)Ia, (cuuint64_t)d.N};
             const cuuint64_t strides[3] = {(cuuint64_t)p.c_w * d.Co * 2, (cuuint64_t)p.c_h * d.Wo * d.Co * 2,
                                            (cuuint64_t)d.Ho * d.Wo * d.Co * 2};
-            const cuuint32_t box[4] = {64, (cuuint32_t)p.Wzq, (cuuint32_t)p.Ic, 1};
+            const cuuint32_t box[4] = {64, (cuuint32_t)p.Wzq, (cuuint32_t)p.rowsB, (cuuint32_t)p.NB};
             const cuuint32_t es[4] = {1, 1, 1, 1};
             char* base = static_cast<char*>(const_cast<void*>(dy)) + ((size_t)a * d.Wo + b) * d.Co * 2;
             if (enc(&p.tmB[a * p.c_w + b], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, es,
