@@ -485,7 +485,8 @@ Tc2Geom build_geom2(const Dims& d) {
     const double mma_clk = up.BN >= 128 ? up.BN / 2.0 : 48.0;   // N = 64 is shared-memory-read bound
     int best_Ic = 0, best_sb = 0, best_NB = 1;
     double best_cost = 1e30, best_eff = 0.0;
-    for (int want = 3; want >= 2 && best_Ic == 0; --want) {
+    {
+        constexpr int want = 2;   // at least two gradient slots; two instead of three costs ~10 %
         for (int Ic = 1; Ic <= I; ++Ic) {
             if (Ic + g.uspan > 256) break;
             for (int NB = 1; NB <= (Ic == I ? 16 : 1) && NB <= d.N; ++NB) {
@@ -502,7 +503,7 @@ Tc2Geom build_geom2(const Dims& d) {
                 const double tiles_per_image = NB == 1 ? (double)bands : 1.0 / NB;
                 const double mmas = (double)U * (KT / 16);
                 const double tile = mmas * mma_clk > 400.0 + 80.0 * mmas ? mmas * mma_clk : 400.0 + 80.0 * mmas;
-                const double cost = tiles_per_image * p.ncls * tile;
+                const double cost = tiles_per_image * p.ncls * tile * (sb < 3 ? 1.1 : 1.0);
                 if (cost < best_cost * (1.0 - 1e-9)) {
                     best_cost = cost; best_Ic = Ic; best_sb = sb; best_NB = NB;
                     best_eff = (double)d.Ho * d.Wo / (tiles_per_image * p.ncls * KT);
