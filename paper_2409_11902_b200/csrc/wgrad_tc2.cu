@@ -39,7 +39,8 @@ using namespace tc;
 
 constexpr int kThreads2 = 192;        // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr int kMaxUnits2 = 8;
-constexpr int kMaxClasses = 16;
+constexpr int kMaxClasses = 64;      // output classes (k/s_h * k/s_w), e.g. k = 8 at stride 1
+constexpr int kMaxClassMaps = 16;    // classes that get a tensor map of their own
 constexpr int kSlotsA = 2;
 constexpr int kMaxSlotsB = 8;
 constexpr uint32_t kSmemBudget2 = 220 * 1024;
@@ -47,7 +48,9 @@ constexpr bool kEnablePairs = true;   // tap pairing for 64-channel layers (plan
 
 struct Tc2Params {
     CUtensorMap tmA;                  // Z as (Ci, Wp, Hp, N)
-    CUtensorMap tmB[kMaxClasses];     // dY, one strided view per class: (Co, J_b, I_a, N)
+    CUtensorMap tmB[kMaxClassMaps];   // dY, one strided view per class: (Co, J_b, I_a, N)
+    CUtensorMap tmBs;                 // more classes than that: dY itself with element strides (c_w, c_h)
+    int strided_map;
     float* out;
     uint32_t* status;
     int Ci, Co, R, S, sh, sw, ph, pw, k;
@@ -67,7 +70,7 @@ struct Tc2Params {
     int pair_mode, pu_count, ncopies;
     int copy_du[3], copy_dv[3];                  // shift of copy g in Z rows / columns
     signed char pu_tapA[kMaxUnits2], pu_tapB[kMaxUnits2];
-    unsigned int pu_off[kMaxClasses][kMaxUnits2];   // A start offset in bytes of (class, unit)
+    unsigned int pu_off[kMaxClassMaps][kMaxUnits2];   // A start offset in bytes of (class, unit)
 };
 
 extern __shared__ __align__(1024) unsigned char tc2_smem[];
@@ -154,9 +157,17 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 if (lane == 0) mbar_arrive_expect_tx(&fullB[sb], (uint32_t)p.nchunks * p.b_box_bytes);
                 __syncwarp();
                 const uint32_t b_slot = b_base + sb * p.b_slot_bytes;
-                if (lane < p.nchunks)
-                    tma_load_4d(b_slot + lane * p.b_chunk_bytes, &p.tmB[pr_cls], &fullB[sb], co0 + 64 * lane, 0,
-                                i0, n);
+                if (lane < p.nchunks) {
+                    if (p.strided_map) {
+                        // one map over dY, traversed with strides (c_w, c_h): the class is the start
+                        const int a = pr_cls / p.c_w, b = pr_cls - a * p.c_w;
+                        tma_load_4d(b_slot + lane * p.b_chunk_bytes, &p.tmBs, &fullB[sb], co0 + 64 * lane, b,
+                                    p.c_h * i0 + a, n);
+                    } else {
+                        tma_load_4d(b_slot + lane * p.b_chunk_bytes, &p.tmB[pr_cls], &fullB[sb],
+                                    co0 + 64 * lane, 0, i0, n);
+                    }
+                }
                 ++pr_tb;
                 if (++pr_cls == p.ncls) { pr_cls = -1; ++pr_kt; ++pr_ta; }
             }
@@ -195,8 +206,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             for (int c = tail0 + lane; c < tail1; c += 32) chunk[c] = zero4;
         }
         fence_proxy_async_smem();
-        const int t2 = tid - 32;
-        if (t2 < p.ncls * kMaxUnits2) {
+        for (int t2 = tid - 32; t2 < p.ncls * kMaxUnits2; t2 += kThreads2 - 32) {
             const int cls = t2 / kMaxUnits2, u = t2 % kMaxUnits2;
             uint32_t off = 0;
             if (p.pair_mode) {
@@ -352,7 +362,8 @@ struct PairPlan {
 bool plan_pairs(const Dims& d, int c_h, int c_w, int umin, int vmin, int uspan, int vspan, PairPlan* out) {
     const int T = d.R * d.S, C = c_h * c_w;
     if (T > 64) return false;
-    static thread_local int ou[kMaxClasses][64], ov[kMaxClasses][64];
+    static thread_local int ou[kMaxClassMaps][64], ov[kMaxClassMaps][64];
+    if (C > kMaxClassMaps) return false;
     for (int c = 0; c < C; ++c)
         for (int t = 0; t < T; ++t) {
             const int a = c / c_w, b = c % c_w, r = t / d.S, sx = t % d.S;
@@ -435,6 +446,7 @@ Tc2Geom build_geom2(const Dims& d) {
     p.c_h = d.k / d.sh; p.c_w = d.k / d.sw;
     p.ncls = p.c_h * p.c_w;
     if (p.ncls > kMaxClasses) return g;
+    p.strided_map = p.ncls > kMaxClassMaps ? 1 : 0;
     if (d.Ho < p.c_h || d.Wo < p.c_w) return g;            // every class has at least one output
     p.Ci = d.Ci; p.Co = d.Co; p.R = d.R; p.S = d.S; p.sh = d.sh; p.sw = d.sw; p.ph = d.ph; p.pw = d.pw;
     p.k = d.k;
@@ -489,6 +501,7 @@ Tc2Geom build_geom2(const Dims& d) {
         constexpr int want = 2;   // at least two gradient slots; two instead of three costs ~10 %
         for (int Ic = 1; Ic <= I; ++Ic) {
             if (Ic + g.uspan > 256) break;
+            if (p.strided_map && (p.c_h * (Ic + g.uspan) > 256 || p.c_w * p.Wzq > 256)) break;
             for (int NB = 1; NB <= (Ic == I ? 16 : 1) && NB <= d.N; ++NB) {
                 const int rowsA = Ic + g.uspan;
                 const int KT = ((NB == 1 ? Ic : NB * rowsA) * p.Wzq + 15) / 16 * 16;
@@ -651,7 +664,19 @@ ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, co
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return AC_ERR_CUDA;
     }
-    for (int a = 0; a < p.c_h; ++a)
+    if (p.strided_map) {
+        const cuuint64_t dims[4] = {(cuuint64_t)d.Co, (cuuint64_t)d.Wo, (cuuint64_t)d.Ho, (cuuint64_t)d.N};
+        const cuuint64_t strides[3] = {(cuuint64_t)d.Co * 2, (cuuint64_t)d.Wo * d.Co * 2,
+                                       (cuuint64_t)d.Ho * d.Wo * d.Co * 2};
+        // the box spans c_w * Wzq columns and c_h * rowsB rows of dY, of which every c_w-th / c_h-th is taken
+        const cuuint32_t box[4] = {64, (cuuint32_t)(p.c_w * p.Wzq), (cuuint32_t)(p.c_h * p.rowsB), (cuuint32_t)p.NB};
+        const cuuint32_t es[4] = {1, (cuuint32_t)p.c_w, (cuuint32_t)p.c_h, 1};
+        if (enc(&p.tmBs, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(dy), dims, strides, box, es,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return AC_ERR_CUDA;
+    }
+    for (int a = 0; a < p.c_h && !p.strided_map; ++a)
         for (int b = 0; b < p.c_w; ++b) {
             // class (a,b): outputs ho = c_h*i + a, wo = c_w*j + b
             const int Ia = (d.Ho - a + p.c_h - 1) / p.c_h, Jb = (d.Wo - b + p.c_w - 1) / p.c_w;
