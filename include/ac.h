@@ -184,15 +184,18 @@ typedef struct {
     int32_t splits;          /* K-slices summed by the split-K reduction */
     int32_t ctas;            /* CTAs of the main kernel */
     int32_t groups;          /* tensor-core path: CTAs that share one K-slice */
-    int32_t band_rows;       /* tensor-core path: output rows per K-tile */
-    int32_t k_tile;          /* tensor-core path: positions per K-tile incl. zero fill */
+    int32_t band_rows;       /* tensor-core path: output rows of one image per K-tile */
+    int32_t k_tile;          /* tensor-core path: positions per K-tile (kernel 2: per class; may span
+                                several whole images of a small map) incl. zero fill */
     int32_t row_pitch;       /* tensor-core path: flat row pitch Wq of the tiles */
     int32_t stages;          /* tensor-core path: shared-memory pipeline depth */
     int32_t smem_bytes;      /* dynamic shared memory per CTA */
     int32_t tmem_columns;    /* tensor-memory columns allocated per CTA */
-    int32_t units_per_cta;   /* tensor-core path: accumulator tiles (128 x block_n) per CTA */
+    int32_t units_per_cta;   /* tensor-core path: accumulator tiles (128 x block_n) per CTA; with 64
+                                input channels a tile may hold two filter taps */
     int32_t block_n;         /* tensor-core path: output channels per accumulator tile */
-    int32_t a_cells;         /* tensor-core path: cells per plane of the inflated input grid */
+    int32_t a_cells;         /* tensor-core path: cells per 64-channel chunk (kernel 2) or per 8-channel
+                                plane (kernel 1) of the input tile in shared memory */
     int32_t phases;          /* tensor-core path: stride phases (kernel 1) or output classes
                                 (kernel 2) per K-tile */
 } ac_plan_info;

@@ -108,13 +108,22 @@ def test_plan_info_respects_hardware_limits(ac):
                 assert i["row_pitch"] >= d.Wo
             else:   # per class: (band_rows / c_h) class rows of row_pitch >= Wo / c_w positions
                 c_h, c_w = k // st, k // st
-                assert i["phases"] == c_h * c_w
+                assert i["phases"] == c_h * c_w <= 64
                 assert i["k_tile"] >= (i["band_rows"] // c_h) * i["row_pitch"]
                 assert i["row_pitch"] >= -(-d.Wo // c_w)
             assert 1 <= i["splits"] <= d.N * -(-d.Ho // i["band_rows"])
             assert i["ctas"] == i["splits"] * i["groups"]
             want = 256 + (i["splits"] * 4 * co * ci * R * S if i["splits"] > 1 else 0)
             assert ac.ac_workspace_bytes(d) == want
+    # 64 input channels, 3x3, k = 2: the nine taps pair up into five accumulator tiles in one CTA
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 64, 64, 56, 56, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
+    assert (i["tensor_core"], i["units_per_cta"], i["groups"]) == (2, 5, 1)
+    # k = 8 at stride 1: 64 output classes, still the TMA-fed kernel
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(256, 128, 128, 64, 64, 3, 3, (1, 1), (1, 1), 8, "bf16", "nhwc"))
+    assert (i["tensor_core"], i["phases"]) == (2, 64)
+    # a map that k does not divide goes to the producer-fed tensor-core kernel
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 512, 512, 7, 7, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
+    assert i["tensor_core"] == 1
     # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
     for d in (ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nhwc"),
               ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
