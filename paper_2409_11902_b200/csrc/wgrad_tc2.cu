@@ -47,7 +47,8 @@ constexpr uint32_t kSmemBudget2 = 220 * 1024;
 constexpr bool kEnablePairs = true;   // tap pairing for 64-channel layers (plan_pairs)
 
 struct Tc2Params {
-    CUtensorMap tmA;                  // Z as (Ci, Wp, Hp, N)
+    CUtensorMap tmA[4];               // Z as (Ci, Wp, Hp, N); variants 1-3 leave out the partial last
+                                      // row and/or column of Z (see `variants` below)
     CUtensorMap tmB[kMaxClassMaps];   // dY, one strided view per class: (Co, J_b, I_a, N)
     CUtensorMap tmBs;                 // more classes than that: dY itself with element strides (c_w, c_h)
     int strided_map;
@@ -62,7 +63,12 @@ struct Tc2Params {
     int taps_per_group, ntapgroups, cibs_per_group, ncibgroups, groups, splits, ktiles;
     int slotsB;
     uint32_t a_slot_bytes, b_slot_bytes, b_chunk_bytes, a_chunk_bytes, a_box_bytes, b_box_bytes, tmem_cols;
-    int chunksA;   // 64-channel chunks of the input tile per slot (incl. one never loaded when CB = 64)
+    int chunksA;   // 64-channel chunks of the input tile per variant (incl. one never loaded when CB = 64)
+    // When k does not divide H (W), the last row (column) of Z is a partial block: it stands for
+    // x in [k*(Hp-1), H) but a tap may also reach the padding rows x in [H, k*Hp), which must read
+    // 0. A (class, tap) pair whose x falls in that second range at the last Z row is served from a
+    // copy of the tile fetched through a tensor map that ends one row (column) earlier.
+    int nvar, var_slot[4], rho_h, rho_w;   // variants in use, variant -> position in the slot, H % k, W % k
     long long dw_elems;
     // Paired mode (64 input channels): one accumulator tile holds TWO taps, rows 0-63
     // tap A and rows 64-127 tap B, because the input tile is kept in up to three copies
@@ -119,7 +125,8 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     // the set-up work below.
     int pr_kt = kt_begin, pr_ta = 0, pr_cls = -1, pr_tb = 0;
     auto produce = [&](bool may_wait) {
-        const int nloads = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);   // 64-channel chunks to fetch
+        const int nchunk_ld = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);   // 64-channel chunks per variant
+        const int nloads = nchunk_ld * p.nvar;
         while (pr_kt < kt_end) {
             const int n = p.NB > 1 ? pr_kt * p.NB : pr_kt / p.bands;
             const int i0 = p.NB > 1 ? 0 : (pr_kt - n * p.bands) * p.Ic;
@@ -137,11 +144,14 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 __syncwarp();
                 const uint32_t a_slot = a_base + sa * p.a_slot_bytes;
                 if (lane < nloads) {
-                    // paired mode: chunk `lane` is copy `lane` of the same 64 channels, shifted
-                    const int ch = p.pair_mode ? 0 : lane * 64;
-                    const int dv = p.pair_mode ? p.copy_dv[lane] : 0, du = p.pair_mode ? p.copy_du[lane] : 0;
-                    tma_load_4d(a_slot + lane * p.a_chunk_bytes, &p.tmA, &fullA[sa], cib0 * p.CB + ch,
-                                p.vmin + dv, i0 + p.umin + du, n);
+                    const int vs = lane / nchunk_ld, c = lane - vs * nchunk_ld;   // variant position, chunk
+                    int var = 0;
+                    for (int v = 0; v < 4; ++v) if (p.var_slot[v] == vs) var = v;
+                    // paired mode: chunk c is copy c of the same 64 channels, shifted
+                    const int ch = p.pair_mode ? 0 : c * 64;
+                    const int dv = p.pair_mode ? p.copy_dv[c] : 0, du = p.pair_mode ? p.copy_du[c] : 0;
+                    tma_load_4d(a_slot + (vs * p.chunksA + c) * p.a_chunk_bytes, &p.tmA[var], &fullA[sa],
+                                cib0 * p.CB + ch, p.vmin + dv, i0 + p.umin + du, n);
                 }
                 pr_cls = 0;
             } else {
@@ -194,9 +204,10 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         const int chunks_real = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);
         const int units16 = (int)(p.a_chunk_bytes / 16), written = p.NB * p.rowsA * p.Wzq * 8;
-        for (int sc = warp - 1; sc < kSlotsA * p.chunksA; sc += kZeroWarps) {
-            const int s_ = sc / p.chunksA, c_ = sc - s_ * p.chunksA;
-            uint4* chunk = reinterpret_cast<uint4*>(smem_gen + (size_t)s_ * p.a_slot_bytes + (size_t)c_ * p.a_chunk_bytes);
+        const int chunks_slot = p.nvar * p.chunksA;
+        for (int sc = warp - 1; sc < kSlotsA * chunks_slot; sc += kZeroWarps) {
+            const int s_ = sc / chunks_slot, cs = sc - s_ * chunks_slot, c_ = cs % p.chunksA;
+            uint4* chunk = reinterpret_cast<uint4*>(smem_gen + (size_t)s_ * p.a_slot_bytes + (size_t)cs * p.a_chunk_bytes);
             for (int c = (c_ < chunks_real ? written : 0) + lane; c < units16; c += 32) chunk[c] = zero4;
         }
         const int tail0 = p.NB * p.rowsB * p.Wzq * 8, tail1 = p.KT * 8;      // in 16-byte units per chunk
@@ -217,7 +228,13 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 const int a = cls / p.c_w, b = cls - a * p.c_w;
                 const int uu = floor_div_i(p.sh * a - p.ph + r, p.k) - p.umin;
                 const int vv = floor_div_i(p.sw * b - p.pw + sx, p.k) - p.vmin;
-                off = (uint32_t)(cl * (p.CB / 64)) * p.a_chunk_bytes + (uint32_t)(uu * p.Wzq + vv) * 128u;
+                // which copy of the tile: the one without the partial last row / column of Z if this
+                // (class, tap) reaches past H / W there
+                const int ch_ = p.sh * a - p.ph + r, cw_ = p.sw * b - p.pw + sx;
+                const int rh = ch_ - floor_div_i(ch_, p.k) * p.k, rw = cw_ - floor_div_i(cw_, p.k) * p.k;
+                const int var = ((p.rho_h > 0 && rh >= p.rho_h) ? 2 : 0) + ((p.rho_w > 0 && rw >= p.rho_w) ? 1 : 0);
+                off = (uint32_t)(p.var_slot[var] * p.chunksA + cl * (p.CB / 64)) * p.a_chunk_bytes +
+                      (uint32_t)(uu * p.Wzq + vv) * 128u;
             }
             aoff_tab[cls][u] = off;
         }
@@ -439,7 +456,6 @@ Tc2Geom build_geom2(const Dims& d) {
     g.ok = false;
     if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
     if (d.k % d.sh != 0 || d.k % d.sw != 0) return g;      // class rows advance Z by exactly one row
-    if (d.H % d.k != 0 || d.W % d.k != 0) return g;        // padding <=> outside the Z tile
     if (d.R * d.S > 64 || d.R > 16 || d.S > 16) return g;
     const UnitPlan up = plan_units(d.Ci, d.Co, d.R * d.S, kMaxUnits2);
     if (!up.ok) return g;
@@ -473,9 +489,24 @@ Tc2Geom build_geom2(const Dims& d) {
     p.cibs_per_group = up.cibs_per_group; p.ncibgroups = up.ncibgroups; p.groups = up.groups;
     p.tmem_cols = up.tmem_cols;
     int chunksA = up.CB == 128 ? 2 * up.cibs_per_group : up.cibs_per_group + 1;
+    // which copies of the Z tile are needed (see Tc2Params::nvar)
+    p.rho_h = d.H % d.k; p.rho_w = d.W % d.k;
+    bool var_used[4] = {false, false, false, false};
+    for (int a = 0; a < p.c_h; ++a)
+        for (int r = 0; r < d.R; ++r)
+            for (int b = 0; b < p.c_w; ++b)
+                for (int s_ = 0; s_ < d.S; ++s_) {
+                    const int ch_ = d.sh * a - d.ph + r, cw_ = d.sw * b - d.pw + s_;
+                    const int rh = ch_ - floor_div_i(ch_, d.k) * d.k, rw = cw_ - floor_div_i(cw_, d.k) * d.k;
+                    var_used[((p.rho_h > 0 && rh >= p.rho_h) ? 2 : 0) + ((p.rho_w > 0 && rw >= p.rho_w) ? 1 : 0)] = true;
+                }
+    p.nvar = 0;
+    for (int v = 0; v < 4; ++v) p.var_slot[v] = var_used[v] ? p.nvar++ : -1;
+    if ((var_used[2] || var_used[3]) && d.Hp < 2) return g;
+    if ((var_used[1] || var_used[3]) && d.Wp < 2) return g;
     PairPlan pairs{};
     p.pair_mode = 0;
-    if (kEnablePairs && d.Ci == 64 && plan_pairs(d, p.c_h, p.c_w, umin, vmin, g.uspan, g.vspan, &pairs) &&
+    if (kEnablePairs && p.nvar == 1 && d.Ci == 64 && plan_pairs(d, p.c_h, p.c_w, umin, vmin, g.uspan, g.vspan, &pairs) &&
         pairs.count * up.BN <= 512) {
         p.pair_mode = 1;
         p.pu_count = pairs.count;
@@ -507,7 +538,7 @@ Tc2Geom build_geom2(const Dims& d) {
                 const int KT = ((NB == 1 ? Ic : NB * rowsA) * p.Wzq + 15) / 16 * 16;
                 const int NCa = (KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
                 if ((uint32_t)NCa * 128 >= (1u << 18) || (uint32_t)KT * 128 >= (1u << 18)) break;
-                const uint32_t a_slot = (uint32_t)chunksA * NCa * 128;
+                const uint32_t a_slot = (uint32_t)p.nvar * chunksA * NCa * 128;
                 const uint32_t b_slot = (uint32_t)p.nchunks * KT * 128;
                 if (kSlotsA * a_slot + want * b_slot > kSmemBudget2) break;
                 int sb = (int)((kSmemBudget2 - kSlotsA * a_slot) / b_slot);
@@ -535,7 +566,7 @@ Tc2Geom build_geom2(const Dims& d) {
     const int NCa = (p.KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
     p.a_chunk_bytes = (uint32_t)NCa * 128;
     p.chunksA = chunksA;
-    p.a_slot_bytes = (uint32_t)chunksA * p.a_chunk_bytes;
+    p.a_slot_bytes = (uint32_t)p.nvar * chunksA * p.a_chunk_bytes;
     if (p.pair_mode) {
         for (int u = 0; u < pairs.count; ++u) {
             p.pu_tapA[u] = (signed char)pairs.tapA[u];
@@ -609,6 +640,8 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
+static_assert(sizeof(Tc2Params) <= 4000, "kernel parameters must stay below the 4 KB limit");
+
 }  // namespace
 
 bool tc2_supported(const Dims& d, double* k_eff) {
@@ -653,13 +686,17 @@ ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, co
     Tc2Params& p = g.p;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return AC_ERR_CUDA;
-    {   // Z viewed as (Ci, Wp, Hp, N); one copy brings 8 channels of a (rows x Wzq) window
-        const cuuint64_t dims[4] = {(cuuint64_t)d.Ci, (cuuint64_t)d.Wp, (cuuint64_t)d.Hp, (cuuint64_t)d.N};
+    for (int var = 0; var < 4; ++var) {
+        if (p.var_slot[var] < 0) continue;
+        // Z viewed as (Ci, Wp, Hp, N); one copy brings 64 channels of a (rows x Wzq) window.
+        // Variants 1-3 end one column and/or one row early: the partial last block reads as zero.
+        const cuuint64_t dims[4] = {(cuuint64_t)d.Ci, (cuuint64_t)(d.Wp - (var & 1)),
+                                    (cuuint64_t)(d.Hp - (var >> 1)), (cuuint64_t)d.N};
         const cuuint64_t strides[3] = {(cuuint64_t)d.Ci * 2, (cuuint64_t)d.Wp * d.Ci * 2,
                                        (cuuint64_t)d.Hp * d.Wp * d.Ci * 2};
         const cuuint32_t box[4] = {64, (cuuint32_t)p.Wzq, (cuuint32_t)p.rowsA, (cuuint32_t)p.NB};
         const cuuint32_t es[4] = {1, 1, 1, 1};
-        if (enc(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(z), dims, strides, box, es,
+        if (enc(&p.tmA[var], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(z), dims, strides, box, es,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return AC_ERR_CUDA;

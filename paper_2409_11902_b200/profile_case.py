@@ -17,6 +17,8 @@ LAYERS = {
     "128ch_28x28": (128, 128, 28, 28, 3, 3, 1, 1),
     "256ch_14x14": (256, 256, 14, 14, 3, 3, 1, 1),
     "512ch_8x8": (512, 512, 8, 8, 3, 3, 1, 1),
+    "512ch_7x7": (512, 512, 7, 7, 3, 3, 1, 1),
+    "2048to512_1x1_7x7": (2048, 512, 7, 7, 1, 1, 1, 0),
     "128ch_64x64": (128, 128, 64, 64, 3, 3, 1, 1),
     "128ch_56x56_s2": (128, 128, 56, 56, 3, 3, 2, 1),
     "256to64_1x1_56x56": (256, 64, 56, 56, 1, 1, 1, 0),

@@ -121,8 +121,11 @@ def test_plan_info_respects_hardware_limits(ac):
     # k = 8 at stride 1: 64 output classes, still the TMA-fed kernel
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(256, 128, 128, 64, 64, 3, 3, (1, 1), (1, 1), 8, "bf16", "nhwc"))
     assert (i["tensor_core"], i["phases"]) == (2, 64)
-    # a map that k does not divide goes to the producer-fed tensor-core kernel
+    # a map that k does not divide (partial pooling blocks) is still taken by the TMA-fed kernel
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 512, 512, 7, 7, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
+    assert i["tensor_core"] == 2
+    # a stride that does not divide k goes to the producer-fed tensor-core kernel
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 28, 28, 3, 3, (2, 2), (1, 1), 1, "bf16", "nhwc"))
     assert i["tensor_core"] == 1
     # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
     for d in (ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nhwc"),
