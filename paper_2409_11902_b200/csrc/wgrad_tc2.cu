@@ -37,7 +37,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads2 = 192;        // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int kThreads2 = 224;        // warp 0: TMA, warps 1 and 6: MMA (1 owns TMEM), warps 2-5: epilogue
+constexpr int kMmaWarps = 2;          // each issues the MMAs of every second accumulator tile
 constexpr int kMaxUnits2 = 8;
 constexpr int kMaxClasses = 64;      // output classes (k/s_h * k/s_w), e.g. k = 8 at stride 1
 constexpr int kMaxClassMaps = 16;    // classes that get a tensor map of their own
@@ -186,9 +187,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], 1); }
-            for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], 1); }
-            mbar_init(&done_bar, 1);
+            for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], kMmaWarps); }
+            for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], kMmaWarps); }
+            mbar_init(&done_bar, kMmaWarps);
             abort_s = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
@@ -247,8 +248,11 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
 
     if (warp == 0) {
         produce(true);
-    } else if (warp == 1) {
-        // ----------------------------------------------------------- MMA issuer
+    } else if (warp == 1 || warp == 6) {
+        // ---------------------------------------------------------- MMA issuers
+        // Two warps, each responsible for every second accumulator tile: the cost of issuing an
+        // MMA (about 80 cycles) is per warp, and tiles are independent.
+        const int mw = warp == 1 ? 0 : 1;
         // The whole warp runs the loop so that the descriptor arithmetic stays in
         // uniform registers; one elected lane issues each MMA and commit.
         const uint32_t idesc = make_idesc(p.BN);
@@ -277,7 +281,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 tc_fence_after();
                 const uint32_t b_lo0 = desc_lo(b_base + sb * p.b_slot_bytes, p.b_chunk_bytes);
                 const uint32_t first = (ta | cls) == 0 ? 0u : 1u;
-                for (int u = 0; u < nunits; ++u) {
+                for (int u = mw; u < nunits; u += kMmaWarps) {
                     // A tap shifts the start by whole 128-byte rows. The swizzle is a function of
                     // the absolute shared-memory address (TMA wrote the tile that way, slots are
                     // 1024-byte aligned), so the descriptor needs no base offset: measured, a
@@ -304,7 +308,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     __syncwarp();
 
     // ---------------------------------------------------------------- epilogue
-    if (warp >= 2) {
+    if (warp >= 2 && warp < 6) {
         bool ok = mbar_wait(&done_bar, 0, abort_flag);
         if (!ok) flag_timeout(&abort_s, p.status, 0x300u);
         ok = __all_sync(0xffffffffu, ok);
