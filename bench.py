@@ -38,6 +38,10 @@ K_POOL = 2
 DTYPE = "bf16"
 LAYOUT = "nhwc"
 N_SETS = 4   # input buffer sets rotated between steps so that inputs are never L2-resident
+# dram__bytes_read.sum + dram__bytes_write.sum of the four wgrad_tc2_kernel launches of one step, from
+# one ncu capture of this command (profiles/launch_list_bench_resnet18_stack.md). Set to None whenever
+# wgrad_tc2.cu changes after that capture.
+WGRAD_DRAM_TRAFFIC_PER_STEP = 61_638_912
 
 
 def load_peaks():
@@ -314,7 +318,12 @@ def run_ours(args):
         "roofline": {"bound": "tensor", "kernel": "ac_conv2d_wgrad_compressed",
                      "achieved": wg_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
                      "frac": wg_tflops / tensor_peak, "peak_source": peaks["source"] + " burst bf16",
-                     "traffic": None},
+                     "traffic": WGRAD_DRAM_TRAFFIC_PER_STEP,
+                     "traffic_unit": "bytes per step (4 launches), ncu",
+                     "algorithmic_bytes": sum((d.N * d.C_in * d.Hp * d.Wp + d.N * d.C_out * d.Ho * d.Wo) * 2
+                                              + d.C_out * d.C_in * d.R * d.S * 4 for _, d in layers),
+                     "step_level": {"achieved": value / world, "frac": value / world / tensor_peak,
+                                    "note": "whole step incl. compress, layers overlapped in the graph"}},
         "e2e": e2e,
         "gpu_launches": args.steps * len(layers) * 3,
         "clocks": clocks,
