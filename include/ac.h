@@ -201,6 +201,16 @@ typedef struct {
 } ac_plan_info;
 ac_status ac_wgrad_plan_info(const ac_conv_desc *desc, ac_plan_info *info);
 
+/*
+ * Self-test of the kernels' failure reporting. Every wait inside the tensor-core kernels is
+ * bounded: when it runs out, the kernel records it in the workspace status block and returns
+ * instead of hanging. This call launches one small kernel that waits, with that same bounded
+ * wait and a limit of `limit_cycles` SM clock cycles (1 .. 2^32), on a barrier nothing will
+ * ever complete. Afterwards ac_workspace_status(workspace) must report AC_ERR_TIMEOUT with
+ * detail 0x7E57. `workspace`: at least 256 bytes of device memory, 16-byte aligned.
+ */
+ac_status ac_selftest_bounded_wait(void *workspace, uint64_t limit_cycles, void *stream);
+
 /* Static, human-readable name of a status code. */
 const char *ac_status_string(ac_status status);
 

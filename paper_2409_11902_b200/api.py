@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.ac_conv2d_wgrad_compressed_static.argtypes = [dp, vp, vp, vp, vp]
         L.ac_wgrad_plan_info.restype = ctypes.c_int
         L.ac_wgrad_plan_info.argtypes = [dp, ctypes.POINTER(ac_plan_info)]
+        L.ac_selftest_bounded_wait.restype = ctypes.c_int
+        L.ac_selftest_bounded_wait.argtypes = [vp, ctypes.c_uint64, vp]
         L.ac_status_string.restype = ctypes.c_char_p
         L.ac_status_string.argtypes = [ctypes.c_int]
         _lib = L
@@ -216,3 +218,9 @@ def ac_wgrad_plan_info(desc: ConvDesc) -> dict:
     if st != AC_OK:
         raise AcError(st, "ac_wgrad_plan_info")
     return {n: getattr(info, n) for n, _ in ac_plan_info._fields_}
+
+
+def ac_selftest_bounded_wait(workspace, limit_cycles: int, stream=None) -> None:
+    st = lib().ac_selftest_bounded_wait(_ptr(workspace), int(limit_cycles), _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_selftest_bounded_wait")

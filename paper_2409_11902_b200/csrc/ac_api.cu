@@ -185,6 +185,14 @@ ac_status ac_wgrad_plan_info(const ac_conv_desc* desc, ac_plan_info* info) {
     return AC_OK;
 }
 
+ac_status ac_selftest_bounded_wait(void* workspace, uint64_t limit_cycles, void* stream) {
+    if (!workspace || limit_cycles == 0 || limit_cycles > (1ull << 32)) return AC_ERR_INVALID_ARG;
+    if (!aligned16(workspace)) return AC_ERR_MISALIGNED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
+    return launch_bounded_wait_selftest(workspace, (long long)limit_cycles, s);
+}
+
 const char* ac_status_string(ac_status status) {
     switch (status) {
         case AC_OK: return "AC_OK";

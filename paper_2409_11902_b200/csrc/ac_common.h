@@ -66,8 +66,22 @@ void plan_tc2(const Dims& d, WgradPlan* p);
 void tc2_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                            float* dw, void* workspace, cudaStream_t stream);
+ac_status launch_bounded_wait_selftest(void* workspace, long long limit_cycles, cudaStream_t stream);
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
                                cudaStream_t stream);
+
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute is per device).
+template <typename Kernel>
+inline ac_status ensure_smem_limit(Kernel kernel, int bytes, bool (&done)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AC_ERR_CUDA;
+    if (!done[dev]) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+            return AC_ERR_CUDA;
+        done[dev] = true;
+    }
+    return AC_OK;
+}
 
 #define AC_CUDA_TRY(expr)                           \
     do {                                            \

@@ -438,11 +438,10 @@ ac_status launch_wgrad_tc(const Dims& d, const WgradPlan& pl, const void* z, con
     p.status = static_cast<uint32_t*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBlockBytes);
     p.out = p.splits > 1 ? partials : dw;
-    static bool attr_set = false;
-    if (!attr_set) {
-        AC_CUDA_TRY(cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kSmemBudget));
-        attr_set = true;
+    static bool attr_done[64] = {};
+    {
+        const ac_status st_ = ensure_smem_limit(wgrad_tc_kernel, (int)kSmemBudget, attr_done);
+        if (st_ != AC_OK) return st_;
     }
     wgrad_tc_kernel<<<p.groups * p.splits, kThreads, g.smem_bytes, stream>>>(p);
     AC_CUDA_TRY(cudaGetLastError());

@@ -357,6 +357,20 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
+// One CTA waits, with the kernels' own bounded wait, on a barrier that nothing will ever
+// complete, and reports it through the workspace status block like the real kernels do.
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, long long limit_cycles) {
+    __shared__ uint64_t never;
+    __shared__ int abort_s;
+    if (threadIdx.x == 0) {
+        mbar_init(&never, 1);
+        abort_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (!mbar_wait(&never, 0, &abort_s, limit_cycles)) flag_timeout(&abort_s, status, 0x7E57u);
+}
+
 // ------------------------------------------------------------------ host side
 struct Tc2Geom {
     Tc2Params p;
@@ -648,6 +662,12 @@ static_assert(sizeof(Tc2Params) <= 4000, "kernel parameters must stay below the 
 
 }  // namespace
 
+ac_status launch_bounded_wait_selftest(void* workspace, long long limit_cycles, cudaStream_t stream) {
+    bounded_wait_selftest_kernel<<<1, 64, 0, stream>>>(static_cast<uint32_t*>(workspace), limit_cycles);
+    AC_CUDA_TRY(cudaGetLastError());
+    return AC_OK;
+}
+
 bool tc2_supported(const Dims& d, double* k_eff) {
     const Tc2Geom g = make_geom2(d);
     if (g.ok && k_eff) *k_eff = g.k_eff;
@@ -735,11 +755,10 @@ ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, co
     p.status = static_cast<uint32_t*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBlockBytes);
     p.out = p.splits > 1 ? partials : dw;
-    static bool attr_set = false;
-    if (!attr_set) {
-        AC_CUDA_TRY(cudaFuncSetAttribute(wgrad_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(kSmemBudget2 + 1024)));
-        attr_set = true;
+    static bool attr_done[64] = {};
+    {
+        const ac_status st_ = ensure_smem_limit(wgrad_tc2_kernel, (int)(kSmemBudget2 + 1024), attr_done);
+        if (st_ != AC_OK) return st_;
     }
     wgrad_tc2_kernel<<<p.groups * p.splits, kThreads2, g.smem_bytes, stream>>>(p);
     AC_CUDA_TRY(cudaGetLastError());

@@ -184,3 +184,19 @@ def test_gradient_alignment_diagnostic():
         assert abs(cos[k] - oracle.cosine_similarity(want, ref)) < 1e-5
     assert cos[1] == pytest.approx(1.0, abs=1e-9)
     assert 0 < cos[4] < cos[2] < 1
+
+
+def test_a_wait_that_runs_out_is_reported_not_hung():
+    """Failure detection without a fault: a kernel waits, with the library's bounded wait, on
+    a barrier that nothing completes; it must come back and leave AC_ERR_TIMEOUT in the status
+    block, and the context must stay usable."""
+    import torch
+    import paper_2409_11902_b200 as ac
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    ac.ac_selftest_bounded_wait(ws, 2_000_000)      # about a millisecond
+    st, detail = ac.ac_workspace_status(ws)
+    assert (st, detail) == (ac.api.AC_ERR_TIMEOUT, 0x7E57)
+    # the device is fine afterwards: an ordinary call still works and reports AC_OK
+    d = D(2, 64, 64, 16, 16, 3, 3, 1, 1, 2, "bf16", "nhwc")
+    z, dy = make_wgrad_inputs(d)
+    run_wgrad(d, z, dy)

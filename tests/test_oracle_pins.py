@@ -353,3 +353,30 @@ def test_ceil_accounting_keeps_partial_blocks():
     assert oracle.compressed_bytes(1, 1, 7, 7, 2, 4, "ceil") == 16 * 4
     assert oracle.compressed_bytes(1, 1, 7, 7, 2, 4, "floor") == 9 * 4
     assert oracle.pool(np.zeros((1, 1, 7, 7)), 2).shape == (1, 1, 4, 4)
+
+
+def test_resnet50_saved_activation_bytes():
+    """Byte accounting for a full ResNet-50 (bottleneck blocks, stride on the 3x3, 224x224
+    images) at batch 256 in bf16, k = 2. Counted per convolution (53 convs, the way the
+    paper's Table 1 lists layers) and per distinct tensor (a block input that feeds both
+    conv1 and the downsample conv is stored once)."""
+    per_conv, unique = [(3, 224)], [(3, 224)]                 # stem
+    # (stage input channels, bottleneck width, output channels, map size at the stage input, blocks, stride)
+    for cin, width, cout, H, blocks, stride in [(64, 64, 256, 56, 3, 1), (256, 128, 512, 56, 4, 2),
+                                                (512, 256, 1024, 28, 6, 2), (1024, 512, 2048, 14, 3, 2)]:
+        for b in range(blocks):
+            h_in = H if b == 0 else H // stride
+            c_in = cin if b == 0 else cout
+            convs = [(c_in, h_in),                                        # conv1 (1x1)
+                     (width, h_in),                                       # conv2 (3x3, carries the stride)
+                     (width, h_in // (stride if b == 0 else 1))]          # conv3 (1x1)
+            per_conv += convs + ([(c_in, h_in)] if b == 0 else [])        # + downsample conv of the first block
+            unique += convs
+    MiB = float(1 << 20)
+    tot = lambda lst, f: sum(f(c, h) for c, h in lst) / MiB
+    xb = lambda c, h: oracle.activation_bytes(256, c, h, h, 2)
+    zb = lambda c, h: oracle.compressed_bytes(256, c, h, h, 2, 2, "ceil")
+    assert len(per_conv) == 53 and len(unique) == 49
+    assert round(tot(per_conv, xb)) == 5206 and round(tot(per_conv, zb)) == 1314
+    assert round(tot(unique, xb)) == 4422 and round(tot(unique, zb)) == 1118
+    assert 0.74 < 1 - tot(unique, zb) / tot(unique, xb) < 0.75
