@@ -202,6 +202,30 @@ typedef struct {
 ac_status ac_wgrad_plan_info(const ac_conv_desc *desc, ac_plan_info *info);
 
 /*
+ * The same weight gradient with the repeated products taken out (the paper's remark that the
+ * compressed form can "reduce the number of memory transactions" taken one step further; Section 4
+ * defines only the result, which is unchanged). Inflation makes neighbouring taps read the same
+ * pooled value: for the outputs of one class (ho mod k/s_h, wo mod k/s_w) every filter tap reads Z
+ * at one of a few distinct shifts, and taps with the same shift form identical products. This call
+ * accumulates one tile per (class, distinct shift) and adds each tile to all taps that map to it:
+ * for a 3x3 filter at k = 2 that is 16 tiles instead of 36, at k = 4 36 instead of 144.
+ * dW equals ac_conv2d_wgrad_compressed's up to fp32 summation order.
+ *
+ * ac_collapsed_workspace_bytes returns the scratch size, or 0 if the problem is not taken in this
+ * form (not bf16/NHWC, channels not multiples of 64, strides not dividing k, k not dividing H and
+ * W, or nothing to collapse such as k = 1 or a 1x1 filter at stride 1); it also reports the number of
+ * accumulated tiles per block of 128 x C_out-block outputs in the collapsed and in the dense
+ * form (their ratio is the saving in tensor-core work). ac_conv2d_wgrad_compressed_collapsed then
+ * returns AC_ERR_UNSUPPORTED for such problems; arguments and conventions are those of
+ * ac_conv2d_wgrad_compressed.
+ */
+size_t ac_collapsed_workspace_bytes(const ac_conv_desc *desc, int32_t *tiles_collapsed,
+                                    int32_t *tiles_dense);
+ac_status ac_conv2d_wgrad_compressed_collapsed(const ac_conv_desc *desc, const void *z,
+                                               const void *dy, float *dw, void *workspace,
+                                               size_t workspace_bytes, void *stream);
+
+/*
  * Self-test of the kernels' failure reporting. Every wait inside the tensor-core kernels is
  * bounded: when it runs out, the kernel records it in the workspace status block and returns
  * instead of hanging. This call launches one small kernel that waits, with that same bounded

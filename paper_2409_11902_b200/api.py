@@ -78,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.ac_wgrad_plan_info.argtypes = [dp, ctypes.POINTER(ac_plan_info)]
         L.ac_selftest_bounded_wait.restype = ctypes.c_int
         L.ac_selftest_bounded_wait.argtypes = [vp, ctypes.c_uint64, vp]
+        L.ac_collapsed_workspace_bytes.restype = sz
+        L.ac_collapsed_workspace_bytes.argtypes = [dp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+        L.ac_conv2d_wgrad_compressed_collapsed.restype = ctypes.c_int
+        L.ac_conv2d_wgrad_compressed_collapsed.argtypes = [dp, vp, vp, vp, vp, sz, vp]
         L.ac_status_string.restype = ctypes.c_char_p
         L.ac_status_string.argtypes = [ctypes.c_int]
         _lib = L
@@ -224,3 +228,23 @@ def ac_selftest_bounded_wait(workspace, limit_cycles: int, stream=None) -> None:
     st = lib().ac_selftest_bounded_wait(_ptr(workspace), int(limit_cycles), _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_selftest_bounded_wait")
+
+
+def ac_collapsed_workspace_bytes(desc: ConvDesc):
+    """(bytes, tiles accumulated in the collapsed form, tiles in the dense form); bytes == 0 if
+    the problem is not taken in the collapsed form."""
+    c = desc.c()
+    a, b = ctypes.c_int32(0), ctypes.c_int32(0)
+    n = int(lib().ac_collapsed_workspace_bytes(ctypes.byref(c), ctypes.byref(a), ctypes.byref(b)))
+    return n, int(a.value), int(b.value)
+
+
+def ac_conv2d_wgrad_compressed_collapsed(desc: ConvDesc, z, dy, dw, workspace, workspace_bytes=None,
+                                         stream=None) -> None:
+    c = desc.c()
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    st = lib().ac_conv2d_wgrad_compressed_collapsed(ctypes.byref(c), _ptr(z), _ptr(dy), _ptr(dw),
+                                                    _ptr(workspace), workspace_bytes, _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_conv2d_wgrad_compressed_collapsed")

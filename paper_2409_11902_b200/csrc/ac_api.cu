@@ -185,6 +185,33 @@ ac_status ac_wgrad_plan_info(const ac_conv_desc* desc, ac_plan_info* info) {
     return AC_OK;
 }
 
+size_t ac_collapsed_workspace_bytes(const ac_conv_desc* desc, int32_t* tiles_collapsed, int32_t* tiles_dense) {
+    Dims d;
+    if (make_dims(desc, true, &d) != AC_OK) return 0;
+    int tc = 0, td = 0;
+    const size_t bytes = tc2_collapsed_workspace_bytes(d, &tc, &td);
+    if (bytes && tiles_collapsed) *tiles_collapsed = tc;
+    if (bytes && tiles_dense) *tiles_dense = td;
+    return bytes;
+}
+
+ac_status ac_conv2d_wgrad_compressed_collapsed(const ac_conv_desc* desc, const void* z, const void* dy,
+                                               float* dw, void* workspace, size_t workspace_bytes,
+                                               void* stream) {
+    Dims d;
+    ac_status st = make_dims(desc, true, &d);
+    if (st != AC_OK) return st;
+    if (!z || !dy || !dw || !workspace) return AC_ERR_INVALID_ARG;
+    if (!aligned16(z) || !aligned16(dy) || !aligned16(dw) || !aligned16(workspace))
+        return AC_ERR_MISALIGNED;
+    const size_t need = tc2_collapsed_workspace_bytes(d, nullptr, nullptr);
+    if (need == 0) return AC_ERR_UNSUPPORTED;
+    if (workspace_bytes < need) return AC_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
+    return launch_wgrad_tc2_collapsed(d, z, dy, dw, workspace, s);
+}
+
 ac_status ac_selftest_bounded_wait(void* workspace, uint64_t limit_cycles, void* stream) {
     if (!workspace || limit_cycles == 0 || limit_cycles > (1ull << 32)) return AC_ERR_INVALID_ARG;
     if (!aligned16(workspace)) return AC_ERR_MISALIGNED;

@@ -66,6 +66,9 @@ void plan_tc2(const Dims& d, WgradPlan* p);
 void tc2_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                            float* dw, void* workspace, cudaStream_t stream);
+size_t tc2_collapsed_workspace_bytes(const Dims& d, int* tiles_collapsed, int* tiles_dense);
+ac_status launch_wgrad_tc2_collapsed(const Dims& d, const void* z, const void* dy, float* dw,
+                                     void* workspace, cudaStream_t stream);
 ac_status launch_bounded_wait_selftest(void* workspace, long long limit_cycles, cudaStream_t stream);
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
                                cudaStream_t stream);

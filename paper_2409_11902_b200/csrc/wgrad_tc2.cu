@@ -78,7 +78,28 @@ struct Tc2Params {
     int copy_du[3], copy_dv[3];                  // shift of copy g in Z rows / columns
     signed char pu_tapA[kMaxUnits2], pu_tapB[kMaxUnits2];
     unsigned int pu_off[kMaxClassMaps][kMaxUnits2];   // A start offset in bytes of (class, unit)
+    // Collapsed mode: within one output class, taps that read the same shift (u,v) of Z form
+    // the same products, so the class gets one accumulator tile per DISTINCT shift instead of
+    // one per tap. Tiles are numbered class by class (cu_total in all); a CTA owns cu_cap
+    // consecutive ones and loads only the classes they belong to; the partial tensor is indexed
+    // by that number and the reduction adds each tile to every tap that maps to it.
+    int collapse, cu_total, cu_cap;
+    long long slice_elems;   // floats of one K-slice of the partial tensor
 };
+
+// Distinct Z shifts of output class `cls`: rows u0 .. u0+nU-1, columns v0 .. v0+nV-1
+// (u = floor((s_h*a - p_h + r) / k) is non-decreasing in r with steps of 0 or 1).
+struct ClassShifts { int u0, nU, v0, nV; };
+__host__ __device__ inline ClassShifts class_shifts(int cls, int c_w, int sh, int sw, int ph, int pw,
+                                                    int k, int R, int S) {
+    const int a = cls / c_w, b = cls - a * c_w;
+    ClassShifts c;
+    c.u0 = floor_div_i(sh * a - ph, k);
+    c.nU = floor_div_i(sh * a - ph + R - 1, k) - c.u0 + 1;
+    c.v0 = floor_div_i(sw * b - pw, k);
+    c.nV = floor_div_i(sw * b - pw + S - 1, k) - c.v0 + 1;
+    return c;
+}
 
 extern __shared__ __align__(1024) unsigned char tc2_smem[];
 
@@ -96,6 +117,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ uint32_t aoff_tab[kMaxClasses][kMaxUnits2];   // A start offset of (class, unit)
+    __shared__ int unit_cls[kMaxUnits2];                     // collapsed mode: class (minus cls0) of a tile
     volatile int* abort_flag = &abort_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -108,7 +130,24 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     const int ntap = min(p.taps_per_group, RS - tap0);
     const int cib0 = cibg * p.cibs_per_group;
     const int ncib = min(p.cibs_per_group, p.ncib_total - cib0);
-    const int nunits = p.pair_mode ? p.pu_count : ncib * ntap;
+    // collapsed mode: this CTA's tiles are numbers [cj0, cj0 + nunits) of the class-by-class
+    // numbering; they belong to classes [cls0, cls1)
+    int cls0 = 0, cls1 = p.ncls, cj0 = 0, cn = 0;
+    if (p.collapse) {
+        cj0 = tg * p.cu_cap;
+        cn = min(p.cu_cap, p.cu_total - cj0);
+        int base = 0;
+        cls0 = -1;
+        for (int c = 0; c < p.ncls; ++c) {
+            const ClassShifts cs = class_shifts(c, p.c_w, p.sh, p.sw, p.ph, p.pw, p.k, p.R, p.S);
+            const int cnt = cs.nU * cs.nV;
+            if (cls0 < 0 && base + cnt > cj0) cls0 = c;
+            if (base < cj0 + cn) cls1 = c + 1;
+            base += cnt;
+        }
+    }
+    const int ncls_mine = cls1 - cls0;
+    const int nunits = p.collapse ? cn : (p.pair_mode ? p.pu_count : ncib * ntap);
     const int co0 = cob * p.BN;
     const int kt_begin = (int)((long long)p.ktiles * split / p.splits);
     const int kt_end = (int)((long long)p.ktiles * (split + 1) / p.splits);
@@ -169,18 +208,19 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 __syncwarp();
                 const uint32_t b_slot = b_base + sb * p.b_slot_bytes;
                 if (lane < p.nchunks) {
+                    const int cls_id = cls0 + pr_cls;
                     if (p.strided_map) {
                         // one map over dY, traversed with strides (c_w, c_h): the class is the start
-                        const int a = pr_cls / p.c_w, b = pr_cls - a * p.c_w;
+                        const int a = cls_id / p.c_w, b = cls_id - a * p.c_w;
                         tma_load_4d(b_slot + lane * p.b_chunk_bytes, &p.tmBs, &fullB[sb], co0 + 64 * lane, b,
                                     p.c_h * i0 + a, n);
                     } else {
-                        tma_load_4d(b_slot + lane * p.b_chunk_bytes, &p.tmB[pr_cls], &fullB[sb],
+                        tma_load_4d(b_slot + lane * p.b_chunk_bytes, &p.tmB[cls_id], &fullB[sb],
                                     co0 + 64 * lane, 0, i0, n);
                     }
                 }
                 ++pr_tb;
-                if (++pr_cls == p.ncls) { pr_cls = -1; ++pr_kt; ++pr_ta; }
+                if (++pr_cls == ncls_mine) { pr_cls = -1; ++pr_kt; ++pr_ta; }
             }
         }
     };
@@ -218,7 +258,22 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             for (int c = tail0 + lane; c < tail1; c += 32) chunk[c] = zero4;
         }
         fence_proxy_async_smem();
-        for (int t2 = tid - 32; t2 < p.ncls * kMaxUnits2; t2 += kThreads2 - 32) {
+        if (p.collapse && tid == 32) {
+            // tile u = number cj0 + u: find its class and its shift inside the class
+            int base = 0, u = 0;
+            for (int c = 0; c < p.ncls && u < nunits; ++c) {
+                const ClassShifts cs = class_shifts(c, p.c_w, p.sh, p.sw, p.ph, p.pw, p.k, p.R, p.S);
+                const int cnt = cs.nU * cs.nV;
+                while (u < nunits && cj0 + u < base + cnt) {
+                    const int j = cj0 + u - base, iu = j / cs.nV, iv = j - iu * cs.nV;
+                    unit_cls[u] = c - cls0;
+                    aoff_tab[0][u] = (uint32_t)((cs.u0 + iu - p.umin) * p.Wzq + (cs.v0 + iv - p.vmin)) * 128u;
+                    ++u;
+                }
+                base += cnt;
+            }
+        }
+        for (int t2 = tid - 32; !p.collapse && t2 < p.ncls * kMaxUnits2; t2 += kThreads2 - 32) {
             const int cls = t2 / kMaxUnits2, u = t2 % kMaxUnits2;
             uint32_t off = 0;
             if (p.pair_mode) {
@@ -270,7 +325,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 break;
             }
             const uint32_t a_lo0 = desc_lo(a_base + sa * p.a_slot_bytes, p.a_chunk_bytes);
-            for (int cls = 0; cls < p.ncls; ++cls, ++tb) {
+            for (int cls = 0; cls < ncls_mine; ++cls, ++tb) {
                 const int sb = tb % p.slotsB;
                 got = mbar_wait(&fullB[sb], (tb / p.slotsB) & 1, abort_flag);
                 if (!__all_sync(0xffffffffu, got)) {
@@ -280,13 +335,16 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 }
                 tc_fence_after();
                 const uint32_t b_lo0 = desc_lo(b_base + sb * p.b_slot_bytes, p.b_chunk_bytes);
-                const uint32_t first = (ta | cls) == 0 ? 0u : 1u;
+                // a tile starts from zero at its first MMA: the first class of the first K-tile, or,
+                // collapsed, the first K-tile (a collapsed tile belongs to one class only)
+                const uint32_t first = (p.collapse ? ta : (ta | cls)) == 0 ? 0u : 1u;
                 for (int u = mw; u < nunits; u += kMmaWarps) {
+                    if (p.collapse && unit_cls[u] != cls) continue;
                     // A tap shifts the start by whole 128-byte rows. The swizzle is a function of
                     // the absolute shared-memory address (TMA wrote the tile that way, slots are
                     // 1024-byte aligned), so the descriptor needs no base offset: measured, a
                     // non-zero base offset here gives wrong sums, zero gives the oracle's.
-                    uint32_t a_lo = a_lo0 + (aoff_tab[cls][u] >> 4);
+                    uint32_t a_lo = a_lo0 + (aoff_tab[p.collapse ? 0 : cls][u] >> 4);
                     const uint32_t a_hi = a_hi0;
                     uint32_t b_lo = b_lo0;
                     const uint32_t dcol = tmem_base + (uint32_t)u * p.BN;
@@ -316,8 +374,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             tc_fence_after();
             const int quarter = warp & 3;            // the TMEM lanes this warp may read
             const int m = quarter * 32 + lane;       // accumulator row
-            float* dst = p.out + (long long)split * p.dw_elems;
-            const long long cstride = (long long)RS * p.Ci;      // floats between output channels
+            float* dst = p.out + (long long)split * (p.collapse ? p.slice_elems : p.dw_elems);
+            // floats between output channels: dW layout, or collapsed [tile][channel out][channel in]
+            const long long cstride = p.collapse ? (long long)p.CB : (long long)RS * p.Ci;
             const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
             const int chunks_per_unit = p.BN / 32, nchunk = nunits * chunks_per_unit;
             // 32 columns at a time, the next chunk's tcgen05.ld in flight while this one is stored
@@ -333,7 +392,15 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                         if (ch + half + 1 < nchunk)
                             tmem_ld32_issue(lane_base + (uint32_t)((ch + half + 1) * 32), buf[half ^ 1]);
                         int tap, ci;
-                        if (p.pair_mode) {
+                        if (p.collapse) {
+                            if (m < p.CB) {
+                                float* q = dst + ((((long long)cob * p.ncib_total + cib0) * p.cu_total + cj0 + u) *
+                                                      p.BN + cu * 32) * p.CB + m;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) q[j * cstride] = __uint_as_float(buf[half][j]);
+                            }
+                            tap = -1; ci = 0;
+                        } else if (p.pair_mode) {
                             tap = m < 64 ? p.pu_tapA[u] : p.pu_tapB[u];
                             ci = cib0 * p.CB + (m & 63);
                         } else {
@@ -355,6 +422,83 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
+}
+
+// Reduction of the collapsed partial tensor P[slice][co block][ci block][tile][co][ci]:
+//   dW[co][r][s][ci] = sum over classes, sum over K-slices of the tile that tap (r,s) maps to in
+//   that class. One float4 of ci per thread group; SL threads share the (class, slice) pairs,
+// each adding its pairs in order, then the SL running sums are added in index order.
+struct CollapseReduceParams {
+    int splits, ncls, R, S, Ci, CB, BN, ncib_total, cu_total, c_w, sh, sw, ph, pw, k;
+    long long slice_elems, elems4;
+};
+
+template <int SL>
+__global__ void __launch_bounds__(256)
+collapsed_reduce_kernel(const float4* __restrict__ P, CollapseReduceParams q, float4* __restrict__ dw) {
+    constexpr int EL = 256 / SL;
+    extern __shared__ unsigned short jmap[];          // [class][tap] -> tile number
+    __shared__ float4 red[SL > 1 ? SL : 1][EL];
+    const int RS = q.R * q.S;
+    {
+        // tile numbering: class by class, inside a class row-major over its distinct shifts
+        for (int e = threadIdx.x; e < q.ncls * RS; e += 256) {
+            const int cls = e / RS, tap = e - cls * RS, r = tap / q.S, sx = tap - r * q.S;
+            int base = 0;
+            for (int c = 0; c < cls; ++c) {
+                const ClassShifts cs = class_shifts(c, q.c_w, q.sh, q.sw, q.ph, q.pw, q.k, q.R, q.S);
+                base += cs.nU * cs.nV;
+            }
+            const ClassShifts cs = class_shifts(cls, q.c_w, q.sh, q.sw, q.ph, q.pw, q.k, q.R, q.S);
+            const int a = cls / q.c_w, b = cls - a * q.c_w;
+            const int iu = floor_div_i(q.sh * a - q.ph + r, q.k) - cs.u0;
+            const int iv = floor_div_i(q.sw * b - q.pw + sx, q.k) - cs.v0;
+            jmap[e] = (unsigned short)(base + iu * cs.nV + iv);
+        }
+    }
+    __syncthreads();
+    const int e = threadIdx.x % EL, sl = threadIdx.x / EL;
+    const long long i = (long long)blockIdx.x * EL + e;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < q.elems4) {
+        const int ci4n = q.Ci / 4;
+        const int ci = (int)(i % ci4n) * 4;
+        const long long t = i / ci4n;
+        const int tap = (int)(t % RS), co = (int)(t / RS);
+        const int cob = co / q.BN, col = co - cob * q.BN, cib = ci / q.CB, m = ci - cib * q.CB;
+        const long long tile0 = ((long long)cob * q.ncib_total + cib) * q.cu_total;
+        const int pairs = q.ncls * q.splits;
+        for (int pq = sl; pq < pairs; pq += SL) {
+            const int cls = pq / q.splits, sp = pq - cls * q.splits;
+            const long long off = (long long)sp * q.slice_elems +
+                                  ((tile0 + jmap[cls * RS + tap]) * q.BN + col) * q.CB + m;
+            const float4 v = __ldcs(P + off / 4);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+    }
+    if (SL == 1) {
+        if (i < q.elems4) dw[i] = acc;
+        return;
+    }
+    red[sl][e] = acc;
+    __syncthreads();
+    if (sl == 0 && i < q.elems4) {
+        float4 o = red[0][e];
+#pragma unroll
+        for (int j = 1; j < SL; ++j) {
+            const float4 v = red[j][e];
+            o.x += v.x; o.y += v.y; o.z += v.z; o.w += v.w;
+        }
+        dw[i] = o;
+    }
+}
+
+template <int SL>
+void launch_collapsed_reduce(const float* P, const CollapseReduceParams& q, float* dw, cudaStream_t st) {
+    constexpr int EL = 256 / SL;
+    const size_t smem = (size_t)q.ncls * q.R * q.S * sizeof(unsigned short);
+    collapsed_reduce_kernel<SL><<<(unsigned)((q.elems4 + EL - 1) / EL), 256, smem, st>>>(
+        reinterpret_cast<const float4*>(P), q, reinterpret_cast<float4*>(dw));
 }
 
 // One CTA waits, with the kernels' own bounded wait, on a barrier that nothing will ever
@@ -468,7 +612,7 @@ bool plan_pairs(const Dims& d, int c_h, int c_w, int umin, int vmin, int uspan, 
     return found;
 }
 
-Tc2Geom build_geom2(const Dims& d) {
+Tc2Geom build_geom2(const Dims& d, bool collapse) {
     Tc2Geom g{};
     Tc2Params& p = g.p;
     g.ok = false;
@@ -524,7 +668,7 @@ Tc2Geom build_geom2(const Dims& d) {
     if ((var_used[1] || var_used[3]) && d.Wp < 2) return g;
     PairPlan pairs{};
     p.pair_mode = 0;
-    if (kEnablePairs && p.nvar == 1 && d.Ci == 64 && plan_pairs(d, p.c_h, p.c_w, umin, vmin, g.uspan, g.vspan, &pairs) &&
+    if (kEnablePairs && !collapse && p.nvar == 1 && d.Ci == 64 && plan_pairs(d, p.c_h, p.c_w, umin, vmin, g.uspan, g.vspan, &pairs) &&
         pairs.count * up.BN <= 512) {
         p.pair_mode = 1;
         p.pu_count = pairs.count;
@@ -542,8 +686,32 @@ Tc2Geom build_geom2(const Dims& d) {
     // the surplus rows are beyond the class's extent and arrive as zeros). Chosen by a cost
     // model per image: a class tile costs max(MMA time, issue time + fixed turn-around),
     // measured at about 80 cycles per MMA issued and 400 cycles per tile.
-    const int U = p.pair_mode ? pairs.count : up.units;
+    const int U = p.collapse ? p.cu_cap : (p.pair_mode ? pairs.count : up.units);
     const double mma_clk = up.BN >= 128 ? up.BN / 2.0 : 48.0;   // N = 64 is shared-memory-read bound
+    p.collapse = 0;
+    if (collapse) {
+        // one accumulator tile per distinct Z shift of each class; needs every class on one copy of
+        // the tile (k | H and k | W) and something to collapse
+        if (p.nvar != 1) return g;
+        int total = 0;
+        for (int c = 0; c < p.ncls; ++c) {
+            const ClassShifts cs = class_shifts(c, p.c_w, d.sh, d.sw, d.ph, d.pw, d.k, d.R, d.S);
+            total += cs.nU * cs.nV;
+        }
+        if (total >= p.ncls * d.R * d.S || total > 65535 || p.ncls * d.R * d.S > 8192) return g;
+        p.collapse = 1;
+        p.cu_total = total;
+        p.cu_cap = 512 / up.BN < kMaxUnits2 ? 512 / up.BN : kMaxUnits2;
+        if (p.cu_cap > total) p.cu_cap = total;
+        p.ntapgroups = (total + p.cu_cap - 1) / p.cu_cap;
+        p.taps_per_group = d.R * d.S;   // not used for tiles in this mode
+        p.cibs_per_group = 1; p.ncibgroups = up.ncib_total;
+        p.groups = up.ncob * up.ncib_total * p.ntapgroups;
+        chunksA = 2;
+        p.tmem_cols = 32;
+        while (p.tmem_cols < (uint32_t)(p.cu_cap * up.BN)) p.tmem_cols *= 2;
+        p.slice_elems = (long long)up.ncob * up.ncib_total * total * up.BN * up.CB;
+    }
     int best_Ic = 0, best_sb = 0, best_NB = 1;
     double best_cost = 1e30, best_eff = 0.0;
     {
@@ -620,22 +788,23 @@ Tc2Geom build_geom2(const Dims& d) {
 // The geometry is pure arithmetic on the descriptor but not free (the pairing search):
 // the last few descriptors are remembered, so that the planning calls of one
 // ac_conv2d_wgrad_compressed (workspace size, support test, launch) and repeated layers pay once.
-Tc2Geom make_geom2(const Dims& d) {
+Tc2Geom make_geom2(const Dims& d, bool collapse = false) {
     constexpr int kEntries = 16;
     static std::mutex mu;
-    static Dims keys[kEntries];
-    static Tc2Geom vals[kEntries];
-    static int used = 0, next = 0;
+    static Dims keys[2][kEntries];
+    static Tc2Geom vals[2][kEntries];
+    static int used[2] = {0, 0}, next[2] = {0, 0};
+    const int w = collapse ? 1 : 0;
     {
         std::lock_guard<std::mutex> lock(mu);
-        for (int i = 0; i < used; ++i)
-            if (std::memcmp(&keys[i], &d, sizeof(Dims)) == 0) return vals[i];
+        for (int i = 0; i < used[w]; ++i)
+            if (std::memcmp(&keys[w][i], &d, sizeof(Dims)) == 0) return vals[w][i];
     }
-    const Tc2Geom g = build_geom2(d);
+    const Tc2Geom g = build_geom2(d, collapse);
     std::lock_guard<std::mutex> lock(mu);
-    keys[next] = d; vals[next] = g;
-    next = (next + 1) % kEntries;
-    if (used < kEntries) ++used;
+    keys[w][next[w]] = d; vals[w][next[w]] = g;
+    next[w] = (next[w] + 1) % kEntries;
+    if (used[w] < kEntries) ++used[w];
     return g;
 }
 
@@ -703,9 +872,9 @@ void tc2_plan_info(const Dims& d, ac_plan_info* info) {
     info->phases = g.p.ncls;
 }
 
-ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, const void* dy,
-                           float* dw, void* workspace, cudaStream_t stream) {
-    Tc2Geom g = make_geom2(d);
+static ac_status launch_tc2_any(const Dims& d, bool collapse, const void* z, const void* dy, float* dw,
+                                void* workspace, cudaStream_t stream) {
+    Tc2Geom g = make_geom2(d, collapse);
     if (!g.ok) return AC_ERR_UNSUPPORTED;
     Tc2Params& p = g.p;
     EncodeTiledFn enc = encode_fn();
@@ -754,7 +923,7 @@ ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, co
         }
     p.status = static_cast<uint32_t*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBlockBytes);
-    p.out = p.splits > 1 ? partials : dw;
+    p.out = (p.splits > 1 || p.collapse) ? partials : dw;
     static bool attr_done[64] = {};
     {
         const ac_status st_ = ensure_smem_limit(wgrad_tc2_kernel, (int)(kSmemBudget2 + 1024), attr_done);
@@ -762,9 +931,48 @@ ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, co
     }
     wgrad_tc2_kernel<<<p.groups * p.splits, kThreads2, g.smem_bytes, stream>>>(p);
     AC_CUDA_TRY(cudaGetLastError());
+    if (p.collapse) {
+        CollapseReduceParams q;
+        q.splits = p.splits; q.ncls = p.ncls; q.R = d.R; q.S = d.S; q.Ci = d.Ci; q.CB = p.CB; q.BN = p.BN;
+        q.ncib_total = p.ncib_total; q.cu_total = p.cu_total; q.c_w = p.c_w; q.sh = d.sh; q.sw = d.sw;
+        q.ph = d.ph; q.pw = d.pw; q.k = d.k; q.slice_elems = p.slice_elems; q.elems4 = p.dw_elems / 4;
+        const int pairs = p.ncls * p.splits;
+        int sl = 1;
+        while (sl < 32 && q.elems4 * sl < 148 * 1024 && sl * 4 <= pairs) sl *= 2;
+        switch (sl) {
+            case 1: launch_collapsed_reduce<1>(partials, q, dw, stream); break;
+            case 2: launch_collapsed_reduce<2>(partials, q, dw, stream); break;
+            case 4: launch_collapsed_reduce<4>(partials, q, dw, stream); break;
+            case 8: launch_collapsed_reduce<8>(partials, q, dw, stream); break;
+            case 16: launch_collapsed_reduce<16>(partials, q, dw, stream); break;
+            default: launch_collapsed_reduce<32>(partials, q, dw, stream); break;
+        }
+        AC_CUDA_TRY(cudaGetLastError());
+        return AC_OK;
+    }
     if (p.splits > 1) return launch_splitk_reduce(partials, p.splits, p.dw_elems, dw, stream);
-    (void)pl;
     return AC_OK;
+}
+
+ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, const void* dy,
+                           float* dw, void* workspace, cudaStream_t stream) {
+    (void)pl;
+    return launch_tc2_any(d, false, z, dy, dw, workspace, stream);
+}
+
+// Collapsed form: same dW, fewer MMAs (see Tc2Params::collapse). 0 bytes / AC_ERR_UNSUPPORTED when the
+// problem has nothing to collapse or the TMA-fed kernel does not take it.
+size_t tc2_collapsed_workspace_bytes(const Dims& d, int* tiles_collapsed, int* tiles_dense) {
+    const Tc2Geom g = make_geom2(d, true);
+    if (!g.ok) return 0;
+    if (tiles_collapsed) *tiles_collapsed = g.p.cu_total;
+    if (tiles_dense) *tiles_dense = g.p.ncls * d.R * d.S;
+    return kStatusBlockBytes + (size_t)g.p.splits * g.p.slice_elems * 4;
+}
+
+ac_status launch_wgrad_tc2_collapsed(const Dims& d, const void* z, const void* dy, float* dw,
+                                     void* workspace, cudaStream_t stream) {
+    return launch_tc2_any(d, true, z, dy, dw, workspace, stream);
 }
 
 }  // namespace ac

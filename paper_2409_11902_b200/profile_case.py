@@ -34,6 +34,7 @@ def main():
     ap.add_argument("--dtype", default="bf16")
     ap.add_argument("--layout", default="nhwc")
     ap.add_argument("--relu", action="store_true", help="use the fused ReLU+compress form")
+    ap.add_argument("--collapsed", action="store_true", help="time the collapsed weight-gradient entry point too")
     a = ap.parse_args()
     ci, co, H, W, R, S, st, pd = LAYERS[a.layer]
     d = api.ConvDesc(a.batch, ci, co, H, W, R, S, (st, st), (pd, pd), a.k, a.dtype, a.layout)
@@ -45,6 +46,9 @@ def main():
     dw = torch.empty(d.dw_shape, dtype=torch.float32, device=dev)
     ws = torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)
     print("plan:", api.ac_wgrad_plan_info(d))
+    cbytes, tiles_c, tiles_d = api.ac_collapsed_workspace_bytes(d) if a.collapsed else (0, 0, 0)
+    cws = torch.empty(max(cbytes, 256), dtype=torch.uint8, device=dev)
+    dwc = torch.empty_like(dw)
     e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
     for it in range(a.iters):
         e0.record()
@@ -55,6 +59,17 @@ def main():
         torch.cuda.synchronize()
         st_, detail = api.ac_workspace_status(ws)
         assert st_ == 0, (st_, detail)
+        if cbytes:
+            e1.record()
+            api.ac_conv2d_wgrad_compressed_collapsed(d, z, dy, dwc, cws)
+            e2.record()
+            torch.cuda.synchronize()
+            ms = e1.elapsed_time(e2)
+            rel = float((dwc - dw).norm() / dw.norm())
+            print(f"iter {it}: collapsed {ms * 1e3:.1f} us: {d.flops / ms / 1e9:.1f} TFLOP/s dense-equivalent, "
+                  f"{d.flops * tiles_c / tiles_d / ms / 1e9:.1f} performed ({tiles_c}/{tiles_d} tiles), "
+                  f"vs dense entry point {rel:.1e}")
+            continue
         print(f"iter {it}: compress {e0.elapsed_time(e1) * 1e3:.1f} us, wgrad {e1.elapsed_time(e2) * 1e3:.1f} us "
               f"({d.flops / e1.elapsed_time(e2) / 1e9:.1f} TFLOP/s)")
 

@@ -137,3 +137,30 @@ def wgrad_error_sampled(d: ac.ConvDesc, n_samples=512, seed=0, dev="cuda:0"):
     g = got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
     assert np.isfinite(got).all()
     return float(np.linalg.norm(g - want) / np.linalg.norm(want)), got
+
+
+def run_wgrad_collapsed(d: ac.ConvDesc, z, dy, dev="cuda:0", repeat=2):
+    """The collapsed entry point, same protocol as run_wgrad. Returns None if the library does
+    not take the problem in that form."""
+    nbytes, tiles_c, tiles_d = ac.ac_collapsed_workspace_bytes(d)
+    if nbytes == 0:
+        return None
+    assert 0 < tiles_c < tiles_d
+    zd = synth.to_layout(z, d.layout).to(dev)
+    dyd = synth.to_layout(dy, d.layout).to(dev)
+    outs = []
+    for it in range(repeat):
+        wbuf, dw, wspan = padded_empty(d.dw_shape, torch.float32, dev)
+        sbuf, ws, sspan = padded_empty((nbytes,), torch.uint8, dev)
+        if it == 1:
+            ws.fill_(0xFF)
+            dw.fill_(float("nan"))
+        ac.ac_conv2d_wgrad_compressed_collapsed(d, zd, dyd, dw, ws, nbytes)
+        st, detail = ac.ac_workspace_status(ws)
+        assert st == 0, f"device status {st} detail {detail:#x}"
+        assert canary_intact(wbuf, wspan), "collapsed wgrad wrote outside dW"
+        assert canary_intact(sbuf, sspan), "collapsed wgrad wrote outside the workspace"
+        outs.append(dw.clone())
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0]), "results differ between identical calls"
+    return dw_to_oihw(outs[0], d.layout)

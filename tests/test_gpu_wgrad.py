@@ -5,7 +5,8 @@ import numpy as np
 import pytest
 
 import __graft_entry__ as entry
-from helpers import TOL_DW, make_wgrad_inputs, run_wgrad, wgrad_error_full, wgrad_error_sampled
+from helpers import (TOL_DW, make_wgrad_inputs, run_wgrad, run_wgrad_collapsed, wgrad_error_full,
+                     wgrad_error_sampled)
 
 pytestmark = pytest.mark.gpu
 
@@ -200,3 +201,55 @@ def test_a_wait_that_runs_out_is_reported_not_hung():
     d = D(2, 64, 64, 16, 16, 3, 3, 1, 1, 2, "bf16", "nhwc")
     z, dy = make_wgrad_inputs(d)
     run_wgrad(d, z, dy)
+
+
+COLLAPSIBLE = [
+    # N, Ci, Co, H, W, R, S, stride, pad, k
+    (2, 64, 64, 16, 16, 3, 3, 1, 1, 2),
+    (3, 128, 128, 12, 20, 3, 3, 1, 1, 2),
+    (2, 128, 64, 16, 16, 3, 3, 2, 1, 2),     # stride 2, k = 2: one class, 4 shifts for 9 taps
+    (2, 64, 128, 16, 16, 3, 3, 1, 1, 4),
+    (2, 128, 128, 16, 16, 3, 3, 1, 1, 8),    # 64 classes
+    (2, 256, 256, 14, 14, 3, 3, 1, 1, 2),
+    (2, 64, 64, 16, 16, 5, 3, 1, 2, 2),
+    (2, 128, 128, 30, 30, 7, 7, 2, 3, 2),
+]
+
+
+@pytest.mark.parametrize("case", COLLAPSIBLE)
+def test_collapsed_form_matches_checker(case):
+    """Fewer MMAs, same dW: against the fp64 checker and against the dense entry point."""
+    import oracle
+    from paper_2409_11902_b200 import synth
+    d = D(*case, "bf16", "nhwc")
+    z, dy = make_wgrad_inputs(d)
+    got = run_wgrad_collapsed(d, z, dy)
+    assert got is not None
+    want = oracle.wgrad_compressed(synth.to_f64(z), synth.to_f64(dy), d.H, d.W, d.R, d.S, d.stride, d.pad, d.k)
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) <= TOL_DW["bf16"]
+    dense = run_wgrad(d, z, dy)
+    assert np.linalg.norm(got - dense) / np.linalg.norm(dense) <= 1e-5
+
+
+def test_collapsed_form_full_size_and_refusals():
+    import paper_2409_11902_b200 as ac
+    import oracle
+    from paper_2409_11902_b200 import synth
+    d = D(64, 128, 128, 28, 28, 3, 3, 1, 1, 2, "bf16", "nhwc")
+    z, dy = make_wgrad_inputs(d)
+    got = run_wgrad_collapsed(d, z, dy)
+    rng = np.random.default_rng(5)
+    idx = np.stack([rng.integers(0, 128, 256), rng.integers(0, 128, 256), rng.integers(0, 3, 256),
+                    rng.integers(0, 3, 256)], axis=1)
+    want = oracle.wgrad_compressed_entries(synth.to_f64(z), synth.to_f64(dy), 28, 28, 3, 3, (1, 1), (1, 1), 2, idx)
+    g = got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
+    assert np.linalg.norm(g - want) / np.linalg.norm(want) <= TOL_DW["bf16"]
+    # nothing to collapse, or not this kernel's shapes: size 0 and AC_ERR_UNSUPPORTED
+    for bad in (D(2, 64, 64, 16, 16, 3, 3, 1, 1, 1, "bf16", "nhwc"), D(2, 64, 64, 16, 16, 1, 1, 1, 0, 2, "bf16", "nhwc"),
+                D(2, 64, 64, 15, 15, 3, 3, 1, 1, 2, "bf16", "nhwc"), D(2, 64, 64, 16, 16, 3, 3, 1, 1, 2, "f32", "nhwc")):
+        assert ac.ac_collapsed_workspace_bytes(bad)[0] == 0
+        import torch
+        t = torch.zeros(1024, device="cuda")
+        with pytest.raises(ac.AcError) as e:
+            ac.ac_conv2d_wgrad_compressed_collapsed(bad, t, t, t, t, 4096)
+        assert e.value.status == ac.api.AC_ERR_UNSUPPORTED
