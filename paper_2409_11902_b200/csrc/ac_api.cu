@@ -107,8 +107,8 @@ ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, co
     const WgradPlan p = plan_wgrad(d);
     if (workspace_bytes < p.bytes) return AC_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (p.path == PATH_TC2) return launch_wgrad_tc2(d, p, z, dy, dw, workspace, s);   // resets the status itself
     AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
-    if (p.path == PATH_TC2) return launch_wgrad_tc2(d, p, z, dy, dw, workspace, s);
     if (p.path == PATH_TC) return launch_wgrad_tc(d, p, z, dy, dw, workspace, s);
     return launch_wgrad_simt(d, p, z, dy, dw, workspace, s);
 }
@@ -208,7 +208,6 @@ ac_status ac_conv2d_wgrad_compressed_collapsed(const ac_conv_desc* desc, const v
     if (need == 0) return AC_ERR_UNSUPPORTED;
     if (workspace_bytes < need) return AC_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
     return launch_wgrad_tc2_collapsed(d, z, dy, dw, workspace, s);
 }
 

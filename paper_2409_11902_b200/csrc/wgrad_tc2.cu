@@ -156,6 +156,10 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     unsigned char* smem_gen = tc2_smem + (smem_base - smem_u32(tc2_smem));
     const uint32_t a_base = smem_base, b_base = smem_base + kSlotsA * p.a_slot_bytes;
 
+    // The status block starts clean: CTA 0 resets it here, long before any wait of this launch
+    // can run out (a wait gives up only after 2^32 cycles).
+    if (blockIdx.x == 0 && tid == 0) { p.status[0] = 0u; p.status[1] = 0u; }
+
     // ---------------------------------------------------------------- TMA producer
     // Warp 0 issues every copy. The stream of copies is: for each K-tile, the Z halo
     // tile (one copy per 8-channel plane, one plane per lane so that the planes of a
