@@ -91,6 +91,26 @@ ac_status ac_compress(const ac_conv_desc *desc, const void *x, void *z,
                       void *y_out, void *stream);
 
 /*
+ * Fused ReLU + compression that keeps a sign mask instead of the activation
+ * (Section 4 replaces the saved conv input by Z; the ReLU in front of it then
+ * needs, for its own backward, only where its input was positive). For a
+ * caller that does not need Y = max(A, 0) in memory afterwards:
+ *
+ *   a     in : the pre-activation A, [N,C_in,H,W] in desc->layout / desc->dtype.
+ *   z     out: pooling of max(A, 0), exactly as ac_compress with y_out writes.
+ *   mask  out: ceil(N*C_in*H*W / 8) bytes on the device; bit (i mod 8) of byte
+ *              (i div 8), least significant bit first, is 1 iff element i of A
+ *              (i counts in memory order of desc->layout) is greater than zero.
+ * The mask is written by the vector kernels only: k must be 1, 2, 4 or 8 and
+ * the contiguous axis (C_in for NHWC; W for NCHW, which k must also divide) a
+ * multiple of 8, k == 1 needs only N*C_in*H*W to be one. Anything else returns
+ * AC_ERR_UNSUPPORTED and launches nothing. All three pointers 16-byte aligned;
+ * one kernel launch on `stream`; no scratch memory.
+ */
+ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z,
+                                void *mask, void *stream);
+
+/*
  * Weight gradient from the compressed activation (Section 4: inflate Z to the
  * original dimensions, then calculate the weight gradient normally; figure:
  * dL/dW ~ Z (*) dL/dY). With Xt[n,c,h,w] = Z[n,c,h/k,w/k] for 0<=h<H, 0<=w<W

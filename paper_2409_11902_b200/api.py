@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.ac_workspace_bytes.argtypes = [dp]
         L.ac_compress.restype = ctypes.c_int
         L.ac_compress.argtypes = [dp, vp, vp, vp, vp]
+        L.ac_compress_relu_mask.restype = ctypes.c_int
+        L.ac_compress_relu_mask.argtypes = [dp, vp, vp, vp, vp]
         L.ac_conv2d_wgrad_compressed.restype = ctypes.c_int
         L.ac_conv2d_wgrad_compressed.argtypes = [dp, vp, vp, vp, vp, sz, vp]
         L.ac_workspace_status.restype = ctypes.c_int
@@ -169,6 +171,13 @@ def ac_compress(desc: ConvDesc, x, z, y_out=None, stream=None) -> None:
     st = lib().ac_compress(ctypes.byref(c), _ptr(x), _ptr(z), _ptr(y_out), _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_compress")
+
+
+def ac_compress_relu_mask(desc: ConvDesc, a, z, mask, stream=None) -> None:
+    c = desc.c()
+    st = lib().ac_compress_relu_mask(ctypes.byref(c), _ptr(a), _ptr(z), _ptr(mask), _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_compress_relu_mask")
 
 
 def ac_conv2d_wgrad_compressed(desc: ConvDesc, z, dy, dw, workspace, workspace_bytes=None,

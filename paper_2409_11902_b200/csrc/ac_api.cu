@@ -95,6 +95,16 @@ ac_status ac_compress(const ac_conv_desc* desc, const void* x, void* z, void* y_
     return launch_compress(d, x, z, y_out, static_cast<cudaStream_t>(stream));
 }
 
+ac_status ac_compress_relu_mask(const ac_conv_desc* desc, const void* a, void* z, void* mask,
+                                void* stream) {
+    Dims d;
+    ac_status st = make_dims(desc, false, &d);
+    if (st != AC_OK) return st;
+    if (!a || !z || !mask) return AC_ERR_INVALID_ARG;
+    if (!aligned16(a) || !aligned16(z) || !aligned16(mask)) return AC_ERR_MISALIGNED;
+    return launch_compress_mask(d, a, z, mask, static_cast<cudaStream_t>(stream));
+}
+
 ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, const void* dy,
                                      float* dw, void* workspace, size_t workspace_bytes,
                                      void* stream) {

@@ -53,6 +53,7 @@ WgradPlan plan_wgrad_simt(const Dims& d);  // the fp32-ALU path's plan, whatever
 
 // ---- launchers (each enqueues on `stream`, returns AC_OK or AC_ERR_CUDA) -----
 ac_status launch_compress(const Dims& d, const void* x, void* z, void* y_out, cudaStream_t stream);
+ac_status launch_compress_mask(const Dims& d, const void* a, void* z, void* mask, cudaStream_t stream);
 ac_status launch_wgrad_simt(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                             float* dw, void* workspace, cudaStream_t stream);
 bool tc_supported(const Dims& d);

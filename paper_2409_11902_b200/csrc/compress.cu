@@ -39,13 +39,15 @@ __device__ __forceinline__ void bf2_to_f(uint32_t u, float& lo, float& hi) {
     lo = __uint_as_float(u << 16);
     hi = __uint_as_float(u & 0xffff0000u);
 }
-// max(x,0) on two packed bf16: clear each half whose sign bit is set
-// (-0 and negative NaN payloads also become +0, like fmaxf(x, 0)).
+// max(x,0) on two packed bf16 in one instruction (-0 and NaN become +0, like fmaxf(x, 0)).
 __device__ __forceinline__ uint32_t relu_bf2(uint32_t u) {
-    uint32_t m = 0;
-    if (!(u & 0x00008000u)) m |= 0x0000ffffu;
-    if (!(u & 0x80000000u)) m |= 0xffff0000u;
-    return u & m;
+    __nv_bfloat162 v = *reinterpret_cast<__nv_bfloat162*>(&u);
+    v = __hmax2(v, __float2bfloat162_rn(0.f));
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// 0xffff in each half of the result whose bf16 is greater than zero
+__device__ __forceinline__ uint32_t positive_bf2(uint32_t u) {
+    return __hgt2_mask(*reinterpret_cast<__nv_bfloat162*>(&u), __float2bfloat162_rn(0.f));
 }
 template <>
 __device__ __forceinline__ void unpack<__nv_bfloat16, false>(uint4& raw, float* f) {
@@ -84,6 +86,38 @@ __device__ __forceinline__ uint4 pack<__nv_bfloat16>(const float* f) {
                       f2_to_bf2(f[6], f[7]));
 }
 
+// Mask mode of the fused form: instead of Y = max(A, 0) the kernel stores one bit per element
+// (1 where A > 0), which is all a ReLU backward needs. Bit i of the mask is element i of A in
+// memory order, least significant bit first. A 16-byte vector is 8 bf16 = one mask byte, or 4
+// fp32 = half a byte: two neighbouring lanes then combine their halves with one shuffle.
+template <typename T>
+__device__ __forceinline__ unsigned positive_bits(const uint4& raw, const float* f);
+template <>
+__device__ __forceinline__ unsigned positive_bits<float>(const uint4&, const float* f) {
+    unsigned b = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) b |= (f[i] > 0.f ? 1u : 0u) << i;
+    return b;
+}
+template <>
+__device__ __forceinline__ unsigned positive_bits<__nv_bfloat16>(const uint4& raw, const float*) {
+    // word j holds elements 2j (low half) and 2j+1 (high half): pick bit 2j of the low
+    // half's flags and bit 16 + 2j + 1 of the high half's, then fold the two halves
+    const unsigned r = (positive_bf2(raw.x) & 0x00020001u) | (positive_bf2(raw.y) & 0x00080004u) |
+                       (positive_bf2(raw.z) & 0x00200010u) | (positive_bf2(raw.w) & 0x00800040u);
+    return (r | (r >> 16)) & 0xffu;
+}
+template <int VW>
+__device__ __forceinline__ void store_mask(unsigned char* mask, long long elem_off, unsigned bits,
+                                           bool valid, unsigned lanes) {
+    if (VW == 8) {
+        if (valid) mask[elem_off >> 3] = (unsigned char)bits;
+    } else {
+        const unsigned other = __shfl_xor_sync(lanes, bits, 1);
+        if (valid && (threadIdx.x & 1) == 0) mask[elem_off >> 3] = (unsigned char)(bits | (other << 4));
+    }
+}
+
 // ---- NHWC, C a multiple of the vector width --------------------------------
 // One thread per output vector (n, p, q, 16 bytes of channels): k*k independent
 // 16-byte loads, element-wise fp32 sums, one 16-byte store. Adjacent threads
@@ -91,13 +125,16 @@ __device__ __forceinline__ uint4 pack<__nv_bfloat16>(const float* f) {
 // Grid: x covers the (q, channel vector) pairs of one pooled row, y = p, z = n,
 // so that no 64-bit division is needed. K > 0: pooling factor known at compile
 // time, all loads of up to four rows issued before the first use; K = 0: any k.
-template <typename T, int K, bool RELU>
+template <typename T, int K, int MODE>   // MODE 0: pool only, 1: also store max(x,0), 2: also store the sign mask
 __global__ void __launch_bounds__(256)
-compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W, int CV, int k,
-                  int Hp, int Wp) {
+compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int CV,
+                  int k, int Hp, int Wp) {
+    constexpr bool RELU = MODE != 0;
     constexpr int VW = VecTraits<T>::VW;
     const unsigned item = blockIdx.x * 256u + threadIdx.x;
-    if (item >= (unsigned)Wp * (unsigned)CV) return;
+    const bool in_range = item < (unsigned)Wp * (unsigned)CV;
+    const unsigned lanes = MODE == 2 ? __ballot_sync(0xffffffffu, in_range) : 0u;   // pairs leave together
+    if (!in_range) return;
     const int q = (int)(item / (unsigned)CV);
     const int cv = (int)(item - (unsigned)q * (unsigned)CV);
     const int p = blockIdx.y;
@@ -120,7 +157,7 @@ compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W
                     const int h = h0 + hb + dh, w = w0 + dw;
                     raw[dh][dw] = make_uint4(0, 0, 0, 0);
                     if (h < h1 && w < w1)
-                        raw[dh][dw] = load16<!RELU>(x + ((((n * H + h) * (long long)W + w) * CV + cv) * VW));
+                        raw[dh][dw] = load16<MODE != 1>(x + ((((n * H + h) * (long long)W + w) * CV + cv) * VW));
                 }
 #pragma unroll
             for (int dh = 0; dh < KR; ++dh) {
@@ -132,9 +169,12 @@ compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W
                     const int h = h0 + hb + dh, w = w0 + dw;
                     float f[VW];
                     unpack<T, RELU>(raw[dh][dw], f);
-                    if (RELU && h < h1 && w < w1)
+                    if (MODE == 1 && h < h1 && w < w1)
                         *reinterpret_cast<uint4*>(y + ((((n * H + h) * (long long)W + w) * CV + cv) * VW)) =
                             raw[dh][dw];
+                    if (MODE == 2)
+                        store_mask<VW>(mask, (((n * H + h) * (long long)W + w) * CV + cv) * VW,
+                                       positive_bits<T>(raw[dh][dw], f), h < h1 && w < w1, lanes);
 #pragma unroll
                     for (int i = 0; i < VW; ++i) row[i] += f[i];
                 }
@@ -150,10 +190,10 @@ compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W
             const long long rbase = ((n * H + h) * (long long)W) * CV + cv;
             for (int w = w0; w < w1; ++w) {
                 const long long off = (rbase + (long long)w * CV) * VW;
-                uint4 raw = load16<!RELU>(x + off);
+                uint4 raw = load16<MODE != 1>(x + off);
                 float f[VW];
                 unpack<T, RELU>(raw, f);
-                if (RELU) *reinterpret_cast<uint4*>(y + off) = raw;
+                if (MODE == 1) *reinterpret_cast<uint4*>(y + off) = raw;
 #pragma unroll
                 for (int i = 0; i < VW; ++i) row[i] += f[i];
             }
@@ -167,18 +207,21 @@ compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W
     *reinterpret_cast<uint4*>(z + ((((n * Hp + p) * (long long)Wp + q) * CV + cv) * VW)) = pack<T>(acc);
 }
 
-template <typename T, bool RELU>
-ac_status launch_nhwc_vec(const T* x, T* z, T* y, long long N, int H, int W, int CV, int k, int Hp, int Wp,
-                          cudaStream_t st) {
+template <typename T, int MODE>
+ac_status launch_nhwc_vec(const T* x, T* z, T* y, unsigned char* mask, long long N, int H, int W, int CV, int k,
+                          int Hp, int Wp, cudaStream_t st) {
     const long long row_items = (long long)Wp * CV;
     if (row_items >= (1ll << 31) || Hp > 65535 || N > 65535) return AC_ERR_UNSUPPORTED;
     dim3 grid((unsigned)((row_items + 255) / 256), (unsigned)Hp, (unsigned)N);
     switch (k) {
-        case 1: compress_nhwc_vec<T, 1, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
-        case 2: compress_nhwc_vec<T, 2, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
-        case 4: compress_nhwc_vec<T, 4, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
-        case 8: compress_nhwc_vec<T, 8, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
-        default: compress_nhwc_vec<T, 0, RELU><<<grid, 256, 0, st>>>(x, z, y, H, W, CV, k, Hp, Wp); break;
+        case 1: compress_nhwc_vec<T, 1, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp); break;
+        case 2: compress_nhwc_vec<T, 2, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp); break;
+        case 4: compress_nhwc_vec<T, 4, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp); break;
+        case 8: compress_nhwc_vec<T, 8, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp); break;
+        default:
+            if (MODE == 2) return AC_ERR_UNSUPPORTED;   // the mask needs warp-uniform loops
+            compress_nhwc_vec<T, 0, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp);
+            break;
     }
     AC_CUDA_TRY(cudaGetLastError());
     return AC_OK;
@@ -189,10 +232,11 @@ ac_status launch_nhwc_vec(const T* x, T* z, T* y, long long N, int H, int W, int
 // read consecutive 16-byte chunks of a row. Vertical sums over the k rows are
 // element-wise; the horizontal sum is a tree inside the vector, finished with
 // one warp shuffle when a block spans two lanes (fp32, k = 8).
-template <typename T, int K, bool RELU, typename I>
+template <typename T, int K, int MODE, typename I>
 __global__ void __launch_bounds__(256)
-compress_nchw_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W, int Hp, int Wp,
-                  long long total) {
+compress_nchw_vec(const T* __restrict__ x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int Hp,
+                  int Wp, long long total) {
+    constexpr bool RELU = MODE != 0;
     constexpr int VW = VecTraits<T>::VW;
     const int WV = W / VW;
     I idx = (I)blockIdx.x * 256u + threadIdx.x;     // I = unsigned when the item count fits 32 bits
@@ -211,15 +255,18 @@ compress_nchw_vec(const T* __restrict__ x, T* __restrict__ z, T* y, int H, int W
 #pragma unroll
     for (int dh = 0; dh < K; ++dh) {
         const int h = h0 + dh;
+        const long long off = ((nc * H + h) * (long long)WV + wv) * VW;
+        unsigned bits = 0;
         if (h < h1) {
-            const long long off = ((nc * H + h) * (long long)WV + wv) * VW;
-            uint4 raw = load16<!RELU>(x + off);
+            uint4 raw = load16<MODE != 1>(x + off);
             float f[VW];
             unpack<T, RELU>(raw, f);
-            if (RELU && active) *reinterpret_cast<uint4*>(y + off) = raw;
+            if (MODE == 1 && active) *reinterpret_cast<uint4*>(y + off) = raw;
+            if (MODE == 2) bits = positive_bits<T>(raw, f);
 #pragma unroll
             for (int i = 0; i < VW; ++i) acc[i] += f[i];
         }
+        if (MODE == 2) store_mask<VW>(mask, off, bits, active && h < h1, 0xffffffffu);
     }
     const float inv = 1.0f / (float)((h1 - h0) * K);
     if (K <= VW) {
@@ -281,40 +328,45 @@ compress_generic(const T* x, T* __restrict__ z, T* y, int C, int H, int W, int k
 
 inline unsigned blocks_for(long long total) { return (unsigned)((total + 255) / 256); }
 
-template <typename T, int K, bool RELU>
-void launch_nchw_vec(const Dims& d, const T* x, T* z, T* y, long long total, cudaStream_t st) {
+template <typename T, int K, int MODE>
+void launch_nchw_vec(const Dims& d, const T* x, T* z, T* y, unsigned char* mask, long long total,
+                     cudaStream_t st) {
     const unsigned g = blocks_for(total);
     if (total < (1ll << 32))
-        compress_nchw_vec<T, K, RELU, unsigned><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp, total);
+        compress_nchw_vec<T, K, MODE, unsigned><<<g, 256, 0, st>>>(x, z, y, mask, d.H, d.W, d.Hp, d.Wp, total);
     else
-        compress_nchw_vec<T, K, RELU, unsigned long long><<<g, 256, 0, st>>>(x, z, y, d.H, d.W, d.Hp, d.Wp,
-                                                                              total);
+        compress_nchw_vec<T, K, MODE, unsigned long long><<<g, 256, 0, st>>>(x, z, y, mask, d.H, d.W, d.Hp,
+                                                                              d.Wp, total);
 }
 
-template <typename T, bool RELU>
-ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, cudaStream_t st) {
+// MODE 2 (sign mask) runs on the vector kernels only: a mask byte covers 8 consecutive elements,
+// so C (NHWC) or W (NCHW) must be a multiple of 8 and k one of 1, 2, 4, 8.
+template <typename T, int MODE>
+ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, unsigned char* mask, cudaStream_t st) {
     constexpr int VW = VecTraits<T>::VW;
     const long long zt = d.z_elems();
     if (zt >= (1ll << 31) * 256) return AC_ERR_UNSUPPORTED;
     const bool pow2k = d.k == 2 || d.k == 4 || d.k == 8;
-    if (d.k == 1 && d.x_elems() % VW == 0) {
+    if (d.k == 1 && d.x_elems() % (MODE == 2 ? 8 : VW) == 0) {
         // a copy (or a plain ReLU): treat the tensor as one row of 16-byte vectors
         const long long nv = d.x_elems() / VW;
         if (nv < (1ll << 31))
-            return launch_nhwc_vec<T, RELU>(x, z, y, 1, 1, (int)nv, 1, 1, 1, (int)nv, st);
+            return launch_nhwc_vec<T, MODE>(x, z, y, mask, 1, 1, (int)nv, 1, 1, 1, (int)nv, st);
     }
-    if (d.layout == AC_NHWC && d.Ci % VW == 0) {
-        const ac_status st_ = launch_nhwc_vec<T, RELU>(x, z, y, d.N, d.H, d.W, d.Ci / VW, d.k, d.Hp, d.Wp, st);
+    if (d.layout == AC_NHWC && d.Ci % (MODE == 2 ? 8 : VW) == 0) {
+        const ac_status st_ =
+            launch_nhwc_vec<T, MODE>(x, z, y, mask, d.N, d.H, d.W, d.Ci / VW, d.k, d.Hp, d.Wp, st);
         if (st_ != AC_ERR_UNSUPPORTED) return st_;
     }
-    if (d.layout == AC_NCHW && pow2k && d.W % VW == 0 && d.W % d.k == 0 &&
+    if (d.layout == AC_NCHW && pow2k && d.W % (MODE == 2 ? 8 : VW) == 0 && d.W % d.k == 0 &&
         (VW % d.k == 0 || d.k == 2 * VW)) {
         const long long total = (long long)d.N * d.Ci * d.Hp * (d.W / VW);
-        if (d.k == 2) launch_nchw_vec<T, 2, RELU>(d, x, z, y, total, st);
-        else if (d.k == 4) launch_nchw_vec<T, 4, RELU>(d, x, z, y, total, st);
-        else launch_nchw_vec<T, 8, RELU>(d, x, z, y, total, st);
+        if (d.k == 2) launch_nchw_vec<T, 2, MODE>(d, x, z, y, mask, total, st);
+        else if (d.k == 4) launch_nchw_vec<T, 4, MODE>(d, x, z, y, mask, total, st);
+        else launch_nchw_vec<T, 8, MODE>(d, x, z, y, mask, total, st);
     } else {
-        compress_generic<T, RELU><<<blocks_for(zt), 256, 0, st>>>(
+        if (MODE == 2) return AC_ERR_UNSUPPORTED;
+        compress_generic<T, MODE != 0><<<blocks_for(zt), 256, 0, st>>>(
             x, z, y, d.Ci, d.H, d.W, d.k, d.Hp, d.Wp, d.layout == AC_NHWC, zt);
     }
     AC_CUDA_TRY(cudaGetLastError());
@@ -325,12 +377,20 @@ ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, cudaStream_t st) {
 
 ac_status launch_compress(const Dims& d, const void* x, void* z, void* y_out, cudaStream_t st) {
     if (d.dtype == AC_F32) {
-        return y_out ? launch_typed<float, true>(d, (const float*)x, (float*)z, (float*)y_out, st)
-                     : launch_typed<float, false>(d, (const float*)x, (float*)z, nullptr, st);
+        return y_out ? launch_typed<float, 1>(d, (const float*)x, (float*)z, (float*)y_out, nullptr, st)
+                     : launch_typed<float, 0>(d, (const float*)x, (float*)z, nullptr, nullptr, st);
     }
     using B = __nv_bfloat16;
-    return y_out ? launch_typed<B, true>(d, (const B*)x, (B*)z, (B*)y_out, st)
-                 : launch_typed<B, false>(d, (const B*)x, (B*)z, nullptr, st);
+    return y_out ? launch_typed<B, 1>(d, (const B*)x, (B*)z, (B*)y_out, nullptr, st)
+                 : launch_typed<B, 0>(d, (const B*)x, (B*)z, nullptr, nullptr, st);
+}
+
+ac_status launch_compress_mask(const Dims& d, const void* a, void* z, void* mask, cudaStream_t st) {
+    if (d.x_elems() % 8 != 0) return AC_ERR_UNSUPPORTED;
+    if (d.dtype == AC_F32)
+        return launch_typed<float, 2>(d, (const float*)a, (float*)z, nullptr, (unsigned char*)mask, st);
+    using B = __nv_bfloat16;
+    return launch_typed<B, 2>(d, (const B*)a, (B*)z, nullptr, (unsigned char*)mask, st);
 }
 
 }  // namespace ac

@@ -34,6 +34,7 @@ def main():
     ap.add_argument("--dtype", default="bf16")
     ap.add_argument("--layout", default="nhwc")
     ap.add_argument("--relu", action="store_true", help="use the fused ReLU+compress form")
+    ap.add_argument("--mask", action="store_true", help="use the fused ReLU+compress form that keeps a sign mask")
     ap.add_argument("--collapsed", action="store_true", help="time the collapsed weight-gradient entry point too")
     a = ap.parse_args()
     ci, co, H, W, R, S, st, pd = LAYERS[a.layer]
@@ -43,6 +44,7 @@ def main():
     dy = synth.to_layout(synth.grad_output(0, (d.N, co, d.Ho, d.Wo), a.dtype), a.layout).to(dev)
     z = torch.empty(d.z_shape, dtype=d.torch_dtype, device=dev)
     y = torch.empty_like(x) if a.relu else None
+    mask = torch.empty((x.numel() + 7) // 8, dtype=torch.uint8, device=dev) if a.mask else None
     dw = torch.empty(d.dw_shape, dtype=torch.float32, device=dev)
     ws = torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)
     print("plan:", api.ac_wgrad_plan_info(d))
@@ -52,7 +54,10 @@ def main():
     e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
     for it in range(a.iters):
         e0.record()
-        api.ac_compress(d, x, z, y)
+        if a.mask:
+            api.ac_compress_relu_mask(d, x, z, mask)
+        else:
+            api.ac_compress(d, x, z, y)
         e1.record()
         api.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws)
         e2.record()

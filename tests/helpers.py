@@ -74,6 +74,29 @@ def run_compress(d: ac.ConvDesc, seed=0, fused_relu=False, inplace=False, dev="c
     return compress_error(z64, x64, d.k), z64, x64
 
 
+def run_compress_mask(d: ac.ConvDesc, seed=0, dev="cuda:0"):
+    """The mask form of the fused call. Returns the pooling error; the mask is compared bit for
+    bit with (A > 0) in memory order."""
+    shape = (d.N, d.C_in, d.H, d.W)
+    a = synth.pre_activation(seed, shape, d.dtype)
+    x64 = oracle.relu(synth.to_f64(a))
+    ad = synth.to_layout(a, d.layout).to(dev)
+    n_el = int(np.prod(shape))
+    zbuf, z, zspan = padded_empty(d.z_shape, d.torch_dtype, dev)
+    mbuf, m, mspan = padded_empty(((n_el + 7) // 8,), torch.uint8, dev)
+    before = ad.clone()
+    ac.ac_compress_relu_mask(d, ad, z, m)
+    torch.cuda.synchronize()
+    assert canary_intact(zbuf, zspan), "wrote outside Z"
+    assert canary_intact(mbuf, mspan), "wrote outside the mask"
+    assert torch.equal(ad.view(torch.uint8), before.view(torch.uint8)), "the input must not be modified"
+    a_mem = synth.to_f64(synth.to_layout(a, d.layout)).reshape(-1)   # memory order of the layout
+    want = np.packbits(a_mem > 0, bitorder="little")
+    assert np.array_equal(m.cpu().numpy(), want), "sign mask differs from (A > 0)"
+    z64 = synth.to_f64(synth.from_layout(z.cpu(), d.layout))
+    return compress_error(z64, x64, d.k)
+
+
 def make_wgrad_inputs(d: ac.ConvDesc, seed=0):
     """X -> Z by the checker's pooling, rounded once to the storage dtype, so
     that the checker and the GPU read identical bits of Z and dY."""

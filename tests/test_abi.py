@@ -64,6 +64,13 @@ def test_calls_validate_before_launching(ac):
     assert L.ac_compress(ref, A + 4, A, None, None) == ac.api.AC_ERR_MISALIGNED
     assert L.ac_compress(ref, A, A, A + 8, None) == ac.api.AC_ERR_MISALIGNED
     assert L.ac_compress(None, A, A, None, None) == ac.api.AC_ERR_INVALID_ARG
+    assert L.ac_compress_relu_mask(ref, A, A, None, None) == ac.api.AC_ERR_INVALID_ARG
+    assert L.ac_compress_relu_mask(ref, A, A, A + 1, None) == ac.api.AC_ERR_MISALIGNED
+    # the sign mask exists only where a mask byte is 8 contiguous elements of a vector kernel
+    for shape in [dict(k=3, layout="nhwc"), dict(k=2, layout="nchw", W=12), dict(k=2, layout="nhwc", C=12)]:
+        m = ac.ConvDesc(2, shape.get("C", 8), 8, 8, shape.get("W", 8), 3, 3, (1, 1), (1, 1), shape["k"],
+                        "bf16", shape["layout"]).c()
+        assert L.ac_compress_relu_mask(ctypes.byref(m), A, A, A, None) == ac.api.AC_ERR_UNSUPPORTED
     assert L.ac_conv2d_wgrad_compressed(ref, A, A, None, A, 1 << 30, None) == ac.api.AC_ERR_INVALID_ARG
     assert L.ac_conv2d_wgrad_compressed(ref, A, A + 2, A, A, 1 << 30, None) == ac.api.AC_ERR_MISALIGNED
     assert L.ac_conv2d_wgrad_compressed(ref, A, A, A, A, 16, None) == ac.api.AC_ERR_WORKSPACE_TOO_SMALL

@@ -2,7 +2,7 @@
 import pytest
 
 import __graft_entry__ as entry
-from helpers import TOL_Z, run_compress
+from helpers import TOL_Z, run_compress, run_compress_mask
 
 pytestmark = pytest.mark.gpu
 
@@ -47,6 +47,33 @@ def test_compress_matches_checker(shape, k, dtype, layout):
 def test_fused_relu_compress(shape, inplace, k, dtype, layout):
     err, _, _ = run_compress(desc(*shape, k, dtype, layout), fused_relu=True, inplace=inplace)
     assert err <= TOL_Z[dtype], err
+
+
+def mask_form_exists(shape, k, layout):
+    """The documented domain of ac_compress_relu_mask."""
+    N, C, H, W = shape
+    if k == 1:
+        return (N * C * H * W) % 8 == 0
+    if layout == "nhwc":
+        return C % 8 == 0
+    return W % 8 == 0 and W % k == 0
+
+
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("k", [1, 2, 3, 4, 8])
+@pytest.mark.parametrize("shape", [(3, 64, 56, 56), (2, 512, 7, 7), (2, 24, 9, 15), (2, 32, 16, 64),
+                                   (2, 16, 9, 16), (1, 3, 16, 24), (1, 3, 17, 23), (5, 8, 3, 40)])
+def test_fused_relu_compress_sign_mask(shape, k, dtype, layout):
+    import paper_2409_11902_b200 as ac
+    d = desc(*shape, k, dtype, layout)
+    if k != 3 and mask_form_exists(shape, k, layout):
+        err = run_compress_mask(d)
+        assert err <= TOL_Z[dtype], err
+    else:
+        with pytest.raises(ac.AcError) as e:
+            run_compress_mask(d)
+        assert e.value.status == ac.api.AC_ERR_UNSUPPORTED
 
 
 def test_large_map_many_blocks():
