@@ -616,6 +616,28 @@ bool plan_pairs(const Dims& d, int c_h, int c_w, int umin, int vmin, int uspan, 
     return found;
 }
 
+// Smallest flat pitch for one axis of the Z tile. The tile holds Z coordinates lo .. lo + P - 1 of
+// every line, lines back to back, and an output at class coordinate c in [0, J) reads coordinate
+// c + v for every shift v in [lo, hi]. A read that runs past the end of its line lands on the first
+// cells of the next one, which is harmless exactly when both the coordinate it wants and the one it
+// gets are outside [0, ext): the tensor map fills those with the convolution's zero padding either
+// way. For a padded 3x3 layer this lets the right halo of one line double as the left halo of the
+// next (P = J + 1 instead of J + 2).
+int min_flat_pitch(int J, int lo, int hi, int ext) {
+    for (int P = J; P < J + (hi - lo); ++P) {
+        bool ok = true;
+        for (int c = 0; c < J && ok; ++c)
+            for (int v = lo; v <= hi && ok; ++v) {
+                const int t = c + v - lo;
+                if (t < P) continue;
+                const int want = c + v, got = lo + t - P;
+                ok = (want < 0 || want >= ext) && (got < 0 || got >= ext) && t - P < P;
+            }
+        if (ok) return P;
+    }
+    return J + (hi - lo);
+}
+
 Tc2Geom build_geom2(const Dims& d, bool collapse) {
     Tc2Geom g{};
     Tc2Params& p = g.p;
@@ -648,6 +670,7 @@ Tc2Geom build_geom2(const Dims& d, bool collapse) {
     g.uspan = umax - umin; g.vspan = vmax - vmin;
     const int I = (d.Ho + p.c_h - 1) / p.c_h, Jc = (d.Wo + p.c_w - 1) / p.c_w;
     p.Wzq = Jc + g.vspan;
+    int rows_whole = I + g.uspan;     // rows per image when a K-tile holds whole images
     if (p.Wzq > 256) return g;
     p.CB = up.CB; p.ncgpc = up.ncgpc; p.ncib_total = up.ncib_total; p.BN = up.BN;
     p.nchunks = up.BN / 64;
@@ -716,6 +739,10 @@ Tc2Geom build_geom2(const Dims& d, bool collapse) {
         while (p.tmem_cols < (uint32_t)(p.cu_cap * up.BN)) p.tmem_cols *= 2;
         p.slice_elems = (long long)up.ncob * up.ncib_total * total * up.BN * up.CB;
     }
+    if (!p.pair_mode && p.nvar == 1) {
+        p.Wzq = min_flat_pitch(Jc, vmin, vmax, d.Wp);
+        rows_whole = min_flat_pitch(I, umin, umax, d.Hp);
+    }
     int best_Ic = 0, best_sb = 0, best_NB = 1;
     double best_cost = 1e30, best_eff = 0.0;
     {
@@ -724,7 +751,7 @@ Tc2Geom build_geom2(const Dims& d, bool collapse) {
             if (Ic + g.uspan > 256) break;
             if (p.strided_map && (p.c_h * (Ic + g.uspan) > 256 || p.c_w * p.Wzq > 256)) break;
             for (int NB = 1; NB <= (Ic == I ? 16 : 1) && NB <= d.N; ++NB) {
-                const int rowsA = Ic + g.uspan;
+                const int rowsA = NB > 1 ? rows_whole : Ic + g.uspan;
                 const int KT = ((NB == 1 ? Ic : NB * rowsA) * p.Wzq + 15) / 16 * 16;
                 const int NCa = (KT + g.uspan * p.Wzq + g.vspan + 7) / 8 * 8;
                 if ((uint32_t)NCa * 128 >= (1u << 18) || (uint32_t)KT * 128 >= (1u << 18)) break;
@@ -749,7 +776,7 @@ Tc2Geom build_geom2(const Dims& d, bool collapse) {
     p.Ic = best_Ic;
     p.NB = best_NB;
     p.bands = (I + p.Ic - 1) / p.Ic;
-    p.rowsA = p.Ic + g.uspan;
+    p.rowsA = p.NB > 1 ? rows_whole : p.Ic + g.uspan;
     p.rowsB = p.NB > 1 ? p.rowsA : p.Ic;
     p.KT = ((p.NB == 1 ? p.Ic : p.NB * p.rowsA) * p.Wzq + 15) / 16 * 16;
     p.ksteps = p.KT / 16;
