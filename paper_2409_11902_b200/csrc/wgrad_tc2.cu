@@ -230,6 +230,15 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     };
 
     if (warp == 0) {
+        // Every tensor map this CTA will use is fetched now, all at once: left to the first copy
+        // that names it, each fetch (about half a microsecond) would hold up the issuing warp in turn.
+        if (lane < 4) {
+            if (p.var_slot[lane] >= 0) prefetch_tmap(&p.tmA[lane]);
+        } else if (p.strided_map) {
+            if (lane == 4) prefetch_tmap(&p.tmBs);
+        } else if (lane - 4 < p.ncls) {
+            prefetch_tmap(&p.tmB[lane - 4]);
+        }
         if (lane == 0) {
             for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], kMmaWarps); }
             for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], kMmaWarps); }
@@ -238,30 +247,38 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         __syncwarp();
-        produce(false);   // fills every slot once; the copies only touch cells no one else writes
+        // The barriers are ready, which is all the other warps need from this one: it reports in
+        // at the set-up barrier without waiting there and goes straight on to issuing copies
+        // (issuing the first round of them takes about 3 us; the first tile lands long before).
+        __threadfence_block();
+        bar_arrive(1, kThreads2);
+        produce(true);
     }
     // Everything the MMAs may read but no copy ever writes must be finite (it only
     // ever meets zeros of the other operand, or feeds accumulator rows that are
     // discarded): the cells behind the last row of each input plane, the planes of
     // the unused upper 64 rows when CB = 64, and the gradient rows behind the tile.
-    if (warp >= 1) {
-        constexpr int kZeroWarps = kThreads2 / 32 - 1;
+    if (warp == 1) tmem_alloc(&tmem_base_s, p.tmem_cols);   // about 0.6 us, beside the zero fill
+    if (warp >= 2) {
+        constexpr int kZeroWarps = kThreads2 / 32 - 2;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         const int chunks_real = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);
         const int units16 = (int)(p.a_chunk_bytes / 16), written = p.NB * p.rowsA * p.Wzq * 8;
         const int chunks_slot = p.nvar * p.chunksA;
-        for (int sc = warp - 1; sc < kSlotsA * chunks_slot; sc += kZeroWarps) {
+        for (int sc = warp - 2; sc < kSlotsA * chunks_slot; sc += kZeroWarps) {
             const int s_ = sc / chunks_slot, cs = sc - s_ * chunks_slot, c_ = cs % p.chunksA;
             uint4* chunk = reinterpret_cast<uint4*>(smem_gen + (size_t)s_ * p.a_slot_bytes + (size_t)cs * p.a_chunk_bytes);
             for (int c = (c_ < chunks_real ? written : 0) + lane; c < units16; c += 32) chunk[c] = zero4;
         }
         const int tail0 = p.NB * p.rowsB * p.Wzq * 8, tail1 = p.KT * 8;      // in 16-byte units per chunk
         unsigned char* bgen = smem_gen + (size_t)kSlotsA * p.a_slot_bytes;
-        for (int sc = warp - 1; sc < p.slotsB * p.nchunks; sc += kZeroWarps) {
+        for (int sc = warp - 2; sc < p.slotsB * p.nchunks; sc += kZeroWarps) {
             uint4* chunk = reinterpret_cast<uint4*>(bgen + (size_t)sc * p.b_chunk_bytes);
             for (int c = tail0 + lane; c < tail1; c += 32) chunk[c] = zero4;
         }
         fence_proxy_async_smem();
+    }
+    if (warp >= 1) {
         if (p.collapse && tid == 32) {
             // tile u = number cj0 + u: find its class and its shift inside the class
             int base = 0, u = 0;
@@ -299,15 +316,15 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             aoff_tab[cls][u] = off;
         }
     }
-    if (warp == 1) tmem_alloc(&tmem_base_s, p.tmem_cols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = tmem_base_s;
+    uint32_t tmem_base = 0;
+    if (warp >= 1) {
+        tc_fence_before();
+        bar_sync(1, kThreads2);
+        tc_fence_after();
+        tmem_base = tmem_base_s;
+    }
 
-    if (warp == 0) {
-        produce(true);
-    } else if (warp == 1 || warp == 6) {
+    if (warp == 1 || warp == 6) {
         // ---------------------------------------------------------- MMA issuers
         // Two warps, each responsible for every second accumulator tile: the cost of issuing an
         // MMA (about 80 cycles) is per warp, and tiles are independent.
