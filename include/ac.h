@@ -119,7 +119,13 @@ ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z
  *   dW[co,ci,r,s] = sum_{n,ho,wo} dY[n,co,ho,wo] * Xt[n,ci,ho*stride_h-pad_h+r,
  *                                                          wo*stride_w-pad_w+s]
  *
- * Xt is never written to memory. Products are accumulated in fp32.
+ * Xt is never written to memory. Products are accumulated in fp32. bf16 inputs
+ * are multiplied exactly (tensor cores); fp32 NHWC inputs that the tensor-core
+ * kernel takes are each split into three bf16 terms and the six leading partial
+ * products are accumulated (terms of relative weight 2^-24 and below are
+ * dropped); the split copies of Z and dY live in the workspace, which is why
+ * ac_workspace_bytes is then about 3 x (|Z| + |dY|) x 4 bytes larger. All other
+ * fp32 problems use fp32 FMA.
  *
  *   z          in : as produced by ac_compress.
  *   dy         in : [N,C_out,H_o,W_o], desc->layout / desc->dtype.
@@ -199,8 +205,10 @@ ac_status ac_conv2d_wgrad_compressed_static(const ac_conv_desc *desc, const void
  * reports and tests). Returns AC_ERR_INVALID_ARG for an invalid descriptor.
  */
 typedef struct {
-    int32_t tensor_core;     /* 2: TMA-fed tcgen05 kernel, 1: tcgen05 kernel with inflating
-                                producer warps, 0: fp32-ALU kernel */
+    int32_t tensor_core;     /* 3: fp32 inputs split into bf16 terms, then as 2 with six times the
+                                images (the other fields describe that launch), 2: TMA-fed tcgen05
+                                kernel, 1: tcgen05 kernel with inflating producer warps,
+                                0: fp32-ALU kernel */
     int32_t splits;          /* K-slices summed by the split-K reduction */
     int32_t ctas;            /* CTAs of the main kernel */
     int32_t groups;          /* tensor-core path: CTAs that share one K-slice */

@@ -65,6 +65,11 @@ WgradPlan plan_wgrad(const Dims& d) {
         plan_tc2(d, &p);
         return p;
     }
+    if (f32x3_supported(d)) {
+        WgradPlan p{};
+        plan_f32x3(d, &p);
+        return p;
+    }
     if (tc_supported(d)) {
         WgradPlan p{};
         p.path = PATH_TC;
@@ -118,6 +123,7 @@ ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, co
     if (workspace_bytes < p.bytes) return AC_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (p.path == PATH_TC2) return launch_wgrad_tc2(d, p, z, dy, dw, workspace, s);   // resets the status itself
+    if (p.path == PATH_F32X3) return launch_wgrad_f32x3(d, p, z, dy, dw, workspace, s);
     AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
     if (p.path == PATH_TC) return launch_wgrad_tc(d, p, z, dy, dw, workspace, s);
     return launch_wgrad_simt(d, p, z, dy, dw, workspace, s);
@@ -181,6 +187,10 @@ ac_status ac_wgrad_plan_info(const ac_conv_desc* desc, ac_plan_info* info) {
     *info = ac_plan_info{};
     if (tc2_supported(d, nullptr)) {
         tc2_plan_info(d, info);
+        return AC_OK;
+    }
+    if (f32x3_supported(d)) {
+        f32x3_plan_info(d, info);
         return AC_OK;
     }
     if (tc_supported(d)) {

@@ -33,7 +33,7 @@ ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* out);
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---- wgrad planning (pure host arithmetic; decides kernel and split-K) ------
-enum WgradPath { PATH_SIMT = 0, PATH_TC = 1, PATH_TC2 = 2 };
+enum WgradPath { PATH_SIMT = 0, PATH_TC = 1, PATH_TC2 = 2, PATH_F32X3 = 3 };
 
 struct WgradPlan {
     int path;        // WgradPath
@@ -45,6 +45,8 @@ struct WgradPlan {
     int tc_groups;   // CTAs sharing one K-slice, each owning part of the output
     int tc_ktiles;   // K-tiles in the whole problem
     int tc_stages;   // shared-memory pipeline depth
+    // fp32 on the tensor cores: where the two split operand tensors sit in the workspace
+    size_t x3_off_z, x3_off_dy;
     size_t bytes;    // workspace bytes including the status block
 };
 
@@ -67,6 +69,12 @@ void plan_tc2(const Dims& d, WgradPlan* p);
 void tc2_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                            float* dw, void* workspace, cudaStream_t stream);
+// fp32 NHWC inputs as six bf16 products on the TMA-fed kernel (wgrad_f32x3.cu)
+bool f32x3_supported(const Dims& d);
+void plan_f32x3(const Dims& d, WgradPlan* p);
+void f32x3_plan_info(const Dims& d, ac_plan_info* info);
+ac_status launch_wgrad_f32x3(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
+                             float* dw, void* workspace, cudaStream_t stream);
 size_t tc2_collapsed_workspace_bytes(const Dims& d, int* tiles_collapsed, int* tiles_dense);
 ac_status launch_wgrad_tc2_collapsed(const Dims& d, const void* z, const void* dy, float* dw,
                                      void* workspace, cudaStream_t stream);

@@ -781,7 +781,12 @@ Tc2Geom build_geom2(const Dims& d, bool collapse) {
                 const double tiles_per_image = NB == 1 ? (double)bands : 1.0 / NB;
                 const double mmas = (double)U * (KT / 16);
                 const double tile = mmas * mma_clk > 400.0 + 80.0 * mmas ? mmas * mma_clk : 400.0 + 80.0 * mmas;
-                const double cost = tiles_per_image * p.ncls * tile * (sb < 3 ? 1.1 : 1.0);
+                // what the slowest CTA does: K-tiles are dealt out whole, so the busiest K-slice
+                // sets the time (448 tiles over 148 slices means 4 for some and 3 for most)
+                const long long kts = NB > 1 ? (d.N + NB - 1) / NB : (long long)d.N * bands;
+                long long spl = kNumSMs / p.groups < 1 ? 1 : kNumSMs / p.groups;
+                if (spl > kts) spl = kts;
+                const double cost = (double)((kts + spl - 1) / spl) * p.ncls * tile * (sb < 3 ? 1.1 : 1.0);
                 if (cost < best_cost * (1.0 - 1e-9)) {
                     best_cost = cost; best_Ic = Ic; best_sb = sb; best_NB = NB;
                     best_eff = (double)d.Ho * d.Wo / (tiles_per_image * p.ncls * KT);

@@ -135,8 +135,18 @@ def test_plan_info_respects_hardware_limits(ac):
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 28, 28, 3, 3, (2, 2), (1, 1), 1, "bf16", "nhwc"))
     assert i["tensor_core"] == 1
     # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
-    for d in (ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nhwc"),
+    for d in (ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw"),
               ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
               ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc"),
               ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (3, 3), (1, 1), 2, "bf16", "nhwc")):
         assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 0
+    # fp32 NHWC goes to the tensor cores as six bf16 products: the same kernel on six times the
+    # images, with room for the split operands in the workspace
+    d32 = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nhwc")
+    d16 = ac.ConvDesc(48, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
+    i32, i16 = ac.ac_wgrad_plan_info(d32), ac.ac_wgrad_plan_info(d16)
+    assert i32["tensor_core"] == 3 and i16["tensor_core"] == 2
+    assert {k: v for k, v in i32.items() if k != "tensor_core"} == {k: v for k, v in i16.items() if k != "tensor_core"}
+    z6 = 48 * 64 * 16 * 16 * 2
+    g6 = 48 * 64 * 32 * 32 * 2
+    assert ac.ac_workspace_bytes(d32) == ac.ac_workspace_bytes(d16) + z6 + g6

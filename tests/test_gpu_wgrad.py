@@ -83,6 +83,18 @@ def test_resnet18_stack_full_size_sampled(N, Ci, Co, H, W):
     assert err <= TOL_DW["bf16"], err
 
 
+@pytest.mark.parametrize("N,Ci,Co,H,W,k", [(64, 128, 128, 28, 28, 2), (64, 64, 64, 56, 56, 2),
+                                             (32, 256, 256, 14, 14, 4), (16, 128, 128, 64, 64, 2)])
+def test_fp32_inputs_on_the_tensor_cores_full_size_sampled(N, Ci, Co, H, W, k):
+    """fp32 NHWC inputs run as six bf16 partial products; the fp32 bound (1e-5) still holds, with
+    at least a factor of two to spare, at sizes where each entry sums 10^4 .. 10^5 products."""
+    import paper_2409_11902_b200 as ac
+    d = D(N, Ci, Co, H, W, 3, 3, 1, 1, k, "f32", "nhwc")
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 3
+    err, _ = wgrad_error_sampled(d, n_samples=256)
+    assert err <= 0.5 * TOL_DW["f32"], err
+
+
 BOTTLENECK = [  # config 3: batch 128, bf16
     (128, 256, 64, 56, 56, 1, 1, 1, 0), (128, 64, 64, 56, 56, 3, 3, 1, 1),
     (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
