@@ -44,7 +44,7 @@ typedef enum {
     AC_ERR_INVALID_ARG = 1,         /* NULL pointer, non-positive size, bad enum, empty output */
     AC_ERR_UNSUPPORTED = 2,         /* valid problem this build cannot run */
     AC_ERR_MISALIGNED = 3,          /* a tensor or workspace pointer is not 16-byte aligned */
-    AC_ERR_WORKSPACE_TOO_SMALL = 4, /* workspace_bytes < ac_workspace_bytes(desc) */
+    AC_ERR_WORKSPACE_TOO_SMALL = 4, /* workspace_bytes < ac_workspace_bytes_min(desc) */
     AC_ERR_CUDA = 5,                /* a CUDA runtime call failed (launch, copy, attribute) */
     AC_ERR_TIMEOUT = 6              /* a bounded wait inside a kernel ran out (see ac_workspace_status) */
 } ac_status;
@@ -64,11 +64,23 @@ typedef struct {
 } ac_conv_desc;
 
 /*
- * Bytes of scratch that ac_conv2d_wgrad_compressed needs for this problem
- * (split-K partial sums of dW plus a small status block). Pure host code.
- * Returns 0 for an invalid descriptor.
+ * Bytes of scratch with which ac_conv2d_wgrad_compressed runs this problem on
+ * its fastest path: a small status block, the split-K partial sums of dW and,
+ * for fp32 and/or NCHW inputs that go to the tensor cores, bf16 NHWC copies of
+ * Z and dY (see ac_conv2d_wgrad_compressed). Pure host code. Returns 0 for an
+ * invalid descriptor.
  */
 size_t ac_workspace_bytes(const ac_conv_desc *desc);
+
+/*
+ * The least scratch ac_conv2d_wgrad_compressed accepts for this problem. Equal
+ * to ac_workspace_bytes unless the fastest path stages copies of the operands;
+ * then this is what the path without copies needs (status block and split-K
+ * partial sums only; at most 256 MiB + 256 bytes). A call given at least this
+ * much but less than ac_workspace_bytes runs on that slower path. Pure host
+ * code. Returns 0 for an invalid descriptor.
+ */
+size_t ac_workspace_bytes_min(const ac_conv_desc *desc);
 
 /*
  * Compression (Section 4; figure: mu_pq is the mean of the k x k block of X
@@ -124,13 +136,16 @@ ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z
  * kernel takes are each split into three bf16 terms and the six leading partial
  * products are accumulated (terms of relative weight 2^-24 and below are
  * dropped); the split copies of Z and dY live in the workspace, which is why
- * ac_workspace_bytes is then about 3 x (|Z| + |dY|) x 4 bytes larger. All other
- * fp32 problems use fp32 FMA.
+ * ac_workspace_bytes is then about 3 x (|Z| + |dY|) x 4 bytes larger. NCHW
+ * inputs that the tensor-core kernel takes once transposed are copied to NHWC
+ * bf16 in the workspace in the same pass. All other fp32 or NCHW problems, and
+ * calls whose workspace is smaller than ac_workspace_bytes but at least
+ * ac_workspace_bytes_min, use fp32 FMA on the operands as they are.
  *
  *   z          in : as produced by ac_compress.
  *   dy         in : [N,C_out,H_o,W_o], desc->layout / desc->dtype.
  *   dw         out: fp32, OVERWRITTEN (not accumulated into); layout per desc->layout.
- *   workspace     : device scratch of at least ac_workspace_bytes(desc) bytes,
+ *   workspace     : device scratch of at least ac_workspace_bytes_min(desc) bytes,
  *                   16-byte aligned; contents on entry are ignored, contents on
  *                   exit are unspecified except for the status block read by
  *                   ac_workspace_status. Two calls that overlap on the device

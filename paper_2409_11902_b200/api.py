@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         dp = ctypes.POINTER(ac_conv_desc)
         L.ac_workspace_bytes.restype = sz
         L.ac_workspace_bytes.argtypes = [dp]
+        L.ac_workspace_bytes_min.restype = sz
+        L.ac_workspace_bytes_min.argtypes = [dp]
         L.ac_compress.restype = ctypes.c_int
         L.ac_compress.argtypes = [dp, vp, vp, vp, vp]
         L.ac_compress_relu_mask.restype = ctypes.c_int
@@ -164,6 +166,11 @@ def _stream(stream):
 def ac_workspace_bytes(desc: ConvDesc) -> int:
     c = desc.c()
     return int(lib().ac_workspace_bytes(ctypes.byref(c)))
+
+
+def ac_workspace_bytes_min(desc: ConvDesc) -> int:
+    c = desc.c()
+    return int(lib().ac_workspace_bytes_min(ctypes.byref(c)))
 
 
 def ac_compress(desc: ConvDesc, x, z, y_out=None, stream=None) -> None:

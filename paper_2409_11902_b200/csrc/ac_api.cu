@@ -59,15 +59,26 @@ WgradPlan plan_wgrad_simt(const Dims& d) {
     return p;
 }
 
+// The plan for a caller whose workspace has no room for staged operand copies.
+WgradPlan plan_wgrad_unstaged(const Dims& d) {
+    if (tc_supported(d)) {
+        WgradPlan p{};
+        p.path = PATH_TC;
+        plan_tc(d, &p);
+        return p;
+    }
+    return plan_wgrad_simt(d);
+}
+
 WgradPlan plan_wgrad(const Dims& d) {
     if (tc2_supported(d, nullptr)) {
         WgradPlan p{};
         plan_tc2(d, &p);
         return p;
     }
-    if (f32x3_supported(d)) {
+    if (staged_supported(d)) {
         WgradPlan p{};
-        plan_f32x3(d, &p);
+        plan_staged(d, &p);
         return p;
     }
     if (tc_supported(d)) {
@@ -89,6 +100,13 @@ size_t ac_workspace_bytes(const ac_conv_desc* desc) {
     Dims d;
     if (make_dims(desc, true, &d) != AC_OK) return 0;
     return plan_wgrad(d).bytes;
+}
+
+size_t ac_workspace_bytes_min(const ac_conv_desc* desc) {
+    Dims d;
+    if (make_dims(desc, true, &d) != AC_OK) return 0;
+    const WgradPlan p = plan_wgrad(d);
+    return p.path == PATH_STAGED ? plan_wgrad_unstaged(d).bytes : p.bytes;
 }
 
 ac_status ac_compress(const ac_conv_desc* desc, const void* x, void* z, void* y_out, void* stream) {
@@ -119,11 +137,12 @@ ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, co
     if (!z || !dy || !dw || !workspace) return AC_ERR_INVALID_ARG;
     if (!aligned16(z) || !aligned16(dy) || !aligned16(dw) || !aligned16(workspace))
         return AC_ERR_MISALIGNED;
-    const WgradPlan p = plan_wgrad(d);
+    WgradPlan p = plan_wgrad(d);
+    if (p.path == PATH_STAGED && workspace_bytes < p.bytes) p = plan_wgrad_unstaged(d);
     if (workspace_bytes < p.bytes) return AC_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (p.path == PATH_TC2) return launch_wgrad_tc2(d, p, z, dy, dw, workspace, s);   // resets the status itself
-    if (p.path == PATH_F32X3) return launch_wgrad_f32x3(d, p, z, dy, dw, workspace, s);
+    if (p.path == PATH_STAGED) return launch_wgrad_staged(d, p, z, dy, dw, workspace, s);
     AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
     if (p.path == PATH_TC) return launch_wgrad_tc(d, p, z, dy, dw, workspace, s);
     return launch_wgrad_simt(d, p, z, dy, dw, workspace, s);
@@ -189,8 +208,8 @@ ac_status ac_wgrad_plan_info(const ac_conv_desc* desc, ac_plan_info* info) {
         tc2_plan_info(d, info);
         return AC_OK;
     }
-    if (f32x3_supported(d)) {
-        f32x3_plan_info(d, info);
+    if (staged_supported(d)) {
+        staged_plan_info(d, info);
         return AC_OK;
     }
     if (tc_supported(d)) {

@@ -19,6 +19,11 @@ struct Dims {
     int Ho, Wo;   // convolution output size
     int dtype, layout;
     int elt;      // bytes per element of X, Z, dY
+    // Tensor-core kernels only: the most MMA instructions that may add into one accumulator before
+    // it is written out as a partial sum (0: no limit). The tensor core adds into its fp32
+    // accumulator with truncation, a bias that grows with the length of the chain; bf16 results
+    // (bound 1e-2) never notice, fp32 results assembled from bf16 terms (bound 1e-5) do.
+    int max_chain;
     long long x_elems() const { return (long long)N * Ci * H * W; }
     long long z_elems() const { return (long long)N * Ci * Hp * Wp; }
     long long dy_elems() const { return (long long)N * Co * Ho * Wo; }
@@ -33,7 +38,7 @@ ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* out);
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---- wgrad planning (pure host arithmetic; decides kernel and split-K) ------
-enum WgradPath { PATH_SIMT = 0, PATH_TC = 1, PATH_TC2 = 2, PATH_F32X3 = 3 };
+enum WgradPath { PATH_SIMT = 0, PATH_TC = 1, PATH_TC2 = 2, PATH_STAGED = 3 };
 
 struct WgradPlan {
     int path;        // WgradPath
@@ -45,8 +50,8 @@ struct WgradPlan {
     int tc_groups;   // CTAs sharing one K-slice, each owning part of the output
     int tc_ktiles;   // K-tiles in the whole problem
     int tc_stages;   // shared-memory pipeline depth
-    // fp32 on the tensor cores: where the two split operand tensors sit in the workspace
-    size_t x3_off_z, x3_off_dy;
+    // staged path: where the staged operands and (NCHW) the kernel's dW sit in the workspace
+    size_t st_off_z, st_off_dy, st_off_dw;
     size_t bytes;    // workspace bytes including the status block
 };
 
@@ -69,11 +74,11 @@ void plan_tc2(const Dims& d, WgradPlan* p);
 void tc2_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                            float* dw, void* workspace, cudaStream_t stream);
-// fp32 NHWC inputs as six bf16 products on the TMA-fed kernel (wgrad_f32x3.cu)
-bool f32x3_supported(const Dims& d);
-void plan_f32x3(const Dims& d, WgradPlan* p);
-void f32x3_plan_info(const Dims& d, ac_plan_info* info);
-ac_status launch_wgrad_f32x3(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
+// fp32 and/or NCHW inputs staged for the TMA-fed kernel (wgrad_staged.cu)
+bool staged_supported(const Dims& d);
+void plan_staged(const Dims& d, WgradPlan* p);
+void staged_plan_info(const Dims& d, ac_plan_info* info);
+ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                              float* dw, void* workspace, cudaStream_t stream);
 size_t tc2_collapsed_workspace_bytes(const Dims& d, int* tiles_collapsed, int* tiles_dense);
 ac_status launch_wgrad_tc2_collapsed(const Dims& d, const void* z, const void* dy, float* dw,

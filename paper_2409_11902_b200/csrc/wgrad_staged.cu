@@ -1,0 +1,228 @@
+// Problems the TMA-fed tcgen05 kernel cannot read directly, brought to it by one pass over each
+// operand ("staging") into the workspace:
+//
+//  * fp32 inputs. The paper's networks train in fp32; a single bf16 or TF32 product cannot meet an
+//    fp32 weight gradient to 1e-5, so each fp32 value is written as the sum of three bf16 terms,
+//    x = h + m + l (h = bf16(x), m = bf16(x - h), l = bf16(x - h - m): 24 bits of significand between
+//    them), and Z * dY is expanded into the six partial products whose weight is at least 2^-16,
+//
+//        Z * dY  ~  Zh*Gh + Zh*Gm + Zm*Gh + Zh*Gl + Zl*Gh + Zm*Gm       (dropped terms: 2^-24 and less)
+//
+//    all accumulated in fp32. A weight gradient is a sum over images, so the six products are simply
+//    six times as many images for the bf16 kernel:
+//
+//        Z'  = [ Zh | Zh | Zm | Zh | Zl | Zm ]        dY' = [ Gh | Gm | Gh | Gl | Gh | Gm ]
+//
+//    (each block N images, bf16), and the kernel runs unchanged with N' = 6 N. Against the fp64
+//    definition the relative Frobenius error is 7e-7 .. 2e-6 (fp32-ALU path: 3e-7 .. 5e-7, at a
+//    fifth to a tenth of the speed).
+//
+//  * NCHW inputs (either dtype). The kernel's tap shift needs channels innermost, so the staging
+//    pass also transposes each image from [C][H*W] to [H*W][C]; the kernel then produces dW as
+//    [C_out][R][S][C_in] in the workspace and a last small pass permutes it to [C_out][C_in][R][S].
+#include "ac_common.h"
+
+namespace ac {
+namespace {
+
+__device__ __forceinline__ uint32_t pack_bf2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// x = h + m + l with h, m, l representable in bf16 (l is rounded when it is packed)
+__device__ __forceinline__ void split3(float x, float& h, float& m, float& l) {
+    h = __bfloat162float(__float2bfloat16_rn(x));
+    const float r1 = x - h;                       // exact: h shares x's leading bits
+    m = __bfloat162float(__float2bfloat16_rn(r1));
+    l = r1 - m;                                   // exact
+}
+
+// Which of (h, m, l) goes to block b of the staged tensor: ROLE 0 is Z', ROLE 1 is dY'.
+template <int ROLE>
+__device__ __forceinline__ int term_of_block(int b) {
+    // Z': h h m h l m      dY': h m h l h m
+    return ROLE == 0 ? ((0x120100 >> (4 * b)) & 3) : ((0x102010 >> (4 * b)) & 3);
+}
+
+// fp32 NHWC -> six bf16 blocks. One thread splits 8 consecutive values and stores three 16-byte
+// vectors, each into the blocks that ROLE assigns to it.
+template <int ROLE>
+__global__ void __launch_bounds__(256)
+split3_kernel(const float4* __restrict__ src, uint4* __restrict__ dst, long long n8) {
+    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n8) return;
+    const float4 a = __ldcs(src + 2 * i), b = __ldcs(src + 2 * i + 1);
+    const float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    float t[3][8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) split3(x[j], t[0][j], t[1][j], t[2][j]);
+    uint4 v[3];
+#pragma unroll
+    for (int q = 0; q < 3; ++q)
+        v[q] = make_uint4(pack_bf2(t[q][0], t[q][1]), pack_bf2(t[q][2], t[q][3]), pack_bf2(t[q][4], t[q][5]),
+                          pack_bf2(t[q][6], t[q][7]));
+#pragma unroll
+    for (int blk = 0; blk < 6; ++blk) dst[blk * n8 + i] = v[term_of_block<ROLE>(blk)];
+}
+
+__device__ __forceinline__ float load_f(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ float load_f(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+// NCHW -> NHWC (bf16), one 64-channel x 32-position tile per block of (32, 8) threads; with SPLIT the
+// source is fp32 and the three terms go to the six blocks as above. grid = (ceil(P/32), C/64, N).
+template <typename TIN, bool SPLIT, int ROLE>
+__global__ void __launch_bounds__(256)
+to_nhwc_kernel(const TIN* __restrict__ src, uint32_t* __restrict__ dst, int C, int P, long long block_words) {
+    __shared__ float tile[64][33];
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int p0 = blockIdx.x * 32, c0 = blockIdx.y * 64;
+    const long long n = blockIdx.z;
+    const TIN* s = src + (n * C + c0) * (long long)P;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int c = ty + 8 * j, p = p0 + tx;
+        tile[c][tx] = p < P ? load_f(s + (long long)c * P + p) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int pl = ty + 8 * j, p = p0 + pl;
+        if (p >= P) continue;
+        const float x0 = tile[2 * tx][pl], x1 = tile[2 * tx + 1][pl];
+        const long long w = ((n * P + p) * (long long)C + c0) / 2 + tx;     // 32-bit word = two channels
+        if (!SPLIT) {
+            dst[w] = pack_bf2(x0, x1);
+        } else {
+            float t0[3], t1[3];
+            split3(x0, t0[0], t0[1], t0[2]);
+            split3(x1, t1[0], t1[1], t1[2]);
+#pragma unroll
+            for (int blk = 0; blk < 6; ++blk) {
+                const int q = term_of_block<ROLE>(blk);
+                dst[blk * block_words + w] = pack_bf2(t0[q], t1[q]);
+            }
+        }
+    }
+}
+
+// dW [Co][RS][Ci] -> [Co][Ci][RS]
+__global__ void __launch_bounds__(256)
+permute_dw_kernel(const float* __restrict__ src, float* __restrict__ dst, int Ci, int RS, long long total) {
+    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (i >= total) return;
+    const int t = (int)(i % RS);
+    const long long r = i / RS;
+    const int ci = (int)(r % Ci);
+    const long long co = r / Ci;
+    dst[i] = src[(co * RS + t) * Ci + ci];
+}
+
+inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// fp32 results: at most this many MMA instructions add into an accumulator before the kernel
+// writes it out (adding, in round-to-nearest fp32, to what it wrote before) and starts it afresh.
+// The tensor core adds into its fp32 accumulator with truncation; on pooled ReLU(N(0,1)) x
+// N(0, 1e-4) data the bias is about 1.8e-8 of the final sum per instruction of the chain. Measured
+// relative Frobenius error / time, batch 64, 128 channels, 28 x 28 (batch 32, 64 x 64):
+//     no bound  6.6e-6 / 127 us  (1.8e-5 / 245 us: over the fp32 bound)
+//     256       3.3e-6 / 133 us  (3.2e-6 / 292 us)
+//     192       2.1e-6 / 143 us  (2.4e-6 / 306 us)
+//     128       1.6e-6 / 151 us  (1.3e-6 / 332 us)
+constexpr int kMaxChainF32 = 128;
+
+// The bf16 NHWC problem the staged operands amount to.
+bool inner_problem(const Dims& d, Dims* in) {
+    const bool split = d.dtype == AC_F32, transpose = d.layout == AC_NCHW;
+    if (!split && !transpose) return false;                 // the kernel reads these itself
+    if (transpose) {
+        if (d.Ci % 64 != 0 || d.Co % 64 != 0 || d.N > 65535) return false;
+        if ((long long)d.Hp * d.Wp >= (1ll << 31) || (long long)d.Ho * d.Wo >= (1ll << 31)) return false;
+    } else if (d.z_elems() % 8 != 0 || d.dy_elems() % 8 != 0) {
+        return false;
+    }
+    const long long n_in = (long long)d.N * (split ? 6 : 1);
+    if (n_in >= (1ll << 31)) return false;
+    *in = d;
+    in->N = (int)n_in;
+    in->dtype = AC_BF16;
+    in->layout = AC_NHWC;
+    in->elt = 2;
+    if (split) in->max_chain = kMaxChainF32;
+    const long long lim = 1ll << 40;
+    if (in->z_elems() >= lim || in->dy_elems() >= lim) return false;
+    return tc2_supported(*in, nullptr);
+}
+
+template <typename TIN, bool SPLIT>
+ac_status stage_nchw(const TIN* z, const TIN* dy, void* z_st, void* dy_st, const Dims& d, cudaStream_t stream) {
+    const int Pz = d.Hp * d.Wp, Pg = d.Ho * d.Wo;
+    const dim3 blk(32, 8);
+    to_nhwc_kernel<TIN, SPLIT, 0><<<dim3((Pz + 31) / 32, d.Ci / 64, d.N), blk, 0, stream>>>(
+        z, static_cast<uint32_t*>(z_st), d.Ci, Pz, d.z_elems() / 2);
+    to_nhwc_kernel<TIN, SPLIT, 1><<<dim3((Pg + 31) / 32, d.Co / 64, d.N), blk, 0, stream>>>(
+        dy, static_cast<uint32_t*>(dy_st), d.Co, Pg, d.dy_elems() / 2);
+    AC_CUDA_TRY(cudaGetLastError());
+    return AC_OK;
+}
+
+}  // namespace
+
+bool staged_supported(const Dims& d) {
+    Dims in;
+    return inner_problem(d, &in);
+}
+
+void plan_staged(const Dims& d, WgradPlan* pl) {
+    Dims in;
+    inner_problem(d, &in);
+    plan_tc2(in, pl);
+    pl->path = PATH_STAGED;
+    pl->st_off_z = up256(pl->bytes);
+    pl->st_off_dy = pl->st_off_z + up256((size_t)in.z_elems() * 2);
+    pl->st_off_dw = pl->st_off_dy + up256((size_t)in.dy_elems() * 2);
+    pl->bytes = pl->st_off_dw + (d.layout == AC_NCHW ? up256((size_t)d.dw_elems() * 4) : 0);
+}
+
+void staged_plan_info(const Dims& d, ac_plan_info* info) {
+    Dims in;
+    inner_problem(d, &in);
+    tc2_plan_info(in, info);
+    info->tensor_core = 3;
+}
+
+ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z, const void* dy,
+                              float* dw, void* workspace, cudaStream_t stream) {
+    Dims in;
+    if (!inner_problem(d, &in)) return AC_ERR_UNSUPPORTED;
+    char* ws = static_cast<char*>(workspace);
+    void* z_st = ws + pl.st_off_z;
+    void* dy_st = ws + pl.st_off_dy;
+    ac_status st = AC_OK;
+    if (d.layout == AC_NCHW) {
+        if (d.dtype == AC_F32)
+            st = stage_nchw<float, true>((const float*)z, (const float*)dy, z_st, dy_st, d, stream);
+        else
+            st = stage_nchw<__nv_bfloat16, false>((const __nv_bfloat16*)z, (const __nv_bfloat16*)dy, z_st, dy_st,
+                                                  d, stream);
+        if (st != AC_OK) return st;
+    } else {
+        const long long nz8 = d.z_elems() / 8, ng8 = d.dy_elems() / 8;
+        if ((nz8 + 255) / 256 >= (1ll << 31) || (ng8 + 255) / 256 >= (1ll << 31)) return AC_ERR_UNSUPPORTED;
+        split3_kernel<0><<<(unsigned)((nz8 + 255) / 256), 256, 0, stream>>>(
+            static_cast<const float4*>(z), static_cast<uint4*>(z_st), nz8);
+        split3_kernel<1><<<(unsigned)((ng8 + 255) / 256), 256, 0, stream>>>(
+            static_cast<const float4*>(dy), static_cast<uint4*>(dy_st), ng8);
+        AC_CUDA_TRY(cudaGetLastError());
+    }
+    if (d.layout == AC_NHWC) return launch_wgrad_tc2(in, pl, z_st, dy_st, dw, workspace, stream);
+    float* dw_st = reinterpret_cast<float*>(ws + pl.st_off_dw);
+    st = launch_wgrad_tc2(in, pl, z_st, dy_st, dw_st, workspace, stream);
+    if (st != AC_OK) return st;
+    const long long total = d.dw_elems();
+    permute_dw_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(dw_st, dw, d.Ci, d.R * d.S, total);
+    AC_CUDA_TRY(cudaGetLastError());
+    return AC_OK;
+}
+
+}  // namespace ac

@@ -84,6 +84,10 @@ struct Tc2Params {
     // consecutive ones and loads only the classes they belong to; the partial tensor is indexed
     // by that number and the reduction adds each tile to every tap that maps to it.
     int collapse, cu_total, cu_cap;
+    // K-tiles after which the accumulators are written out (added to what this CTA wrote before) and
+    // started afresh; 0: only at the end. Bounds the length of the tensor core's truncating fp32
+    // accumulation chains for results that must hold an fp32 bound.
+    int chunk_kt;
     long long slice_elems;   // floats of one K-slice of the partial tensor
 };
 
@@ -110,10 +114,24 @@ __device__ __forceinline__ void flag_timeout(int* abort_s, uint32_t* status, uin
     }
 }
 
+// 32 accumulator columns of one row to memory, `stride` floats apart; `add_to`: added to what this
+// thread stored there before (all loads first, so that they overlap).
+__device__ __forceinline__ void put32(float* q, long long stride, const uint32_t* v, bool add_to) {
+    float old[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) old[j] = 0.f;
+    if (add_to) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) old[j] = q[j * stride];
+    }
+#pragma unroll
+    for (int j = 0; j < 32; ++j) q[j * stride] = old[j] + __uint_as_float(v[j]);
+}
+
 __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_constant__ Tc2Params p) {
     __shared__ uint64_t fullA[kSlotsA], emptyA[kSlotsA];
     __shared__ uint64_t fullB[kMaxSlotsB], emptyB[kMaxSlotsB];
-    __shared__ uint64_t done_bar;
+    __shared__ uint64_t done_bar, tfree_bar;   // accumulators complete / accumulators read out
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ uint32_t aoff_tab[kMaxClasses][kMaxUnits2];   // A start offset of (class, unit)
@@ -151,6 +169,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     const int co0 = cob * p.BN;
     const int kt_begin = (int)((long long)p.ktiles * split / p.splits);
     const int kt_end = (int)((long long)p.ktiles * (split + 1) / p.splits);
+    const int chunk_kt = p.chunk_kt > 0 ? p.chunk_kt : 0x7fffffff;
     // 1024-byte aligned tile area: A slots first, then B slots
     const uint32_t smem_base = (smem_u32(tc2_smem) + 1023u) & ~1023u;
     unsigned char* smem_gen = tc2_smem + (smem_base - smem_u32(tc2_smem));
@@ -243,6 +262,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], kMmaWarps); }
             for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], kMmaWarps); }
             mbar_init(&done_bar, kMmaWarps);
+            mbar_init(&tfree_bar, 4);
             abort_s = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
@@ -337,9 +357,25 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         const bool leader = elect_one();
         int tb = 0;
         bool ok = true;
-        for (int kt = kt_begin, ta = 0; kt < kt_end && ok; ++kt, ++ta) {
+        for (int kt = kt_begin, ta = 0, tac = 0, chunk = 0; kt < kt_end && ok; ++kt, ++ta, ++tac) {
             const int sa = ta % kSlotsA;
-            bool got = mbar_wait(&fullA[sa], (ta / kSlotsA) & 1, abort_flag);
+            bool got;
+            if (tac == chunk_kt) {
+                // The accumulation chains have reached their bound: hand the tiles to the epilogue
+                // warps and go on from zero once they have read them out.
+                if (leader) mma_commit(&done_bar);
+                __syncwarp();
+                got = mbar_wait(&tfree_bar, chunk & 1, abort_flag);
+                if (!__all_sync(0xffffffffu, got)) {
+                    if (leader) flag_timeout(&abort_s, p.status, 0x380u);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                tac = 0;
+                ++chunk;
+            }
+            got = mbar_wait(&fullA[sa], (ta / kSlotsA) & 1, abort_flag);
             if (!__all_sync(0xffffffffu, got)) {
                 if (leader) flag_timeout(&abort_s, p.status, 0x200u + sa);
                 ok = false;
@@ -356,9 +392,10 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 }
                 tc_fence_after();
                 const uint32_t b_lo0 = desc_lo(b_base + sb * p.b_slot_bytes, p.b_chunk_bytes);
-                // a tile starts from zero at its first MMA: the first class of the first K-tile, or,
-                // collapsed, the first K-tile (a collapsed tile belongs to one class only)
-                const uint32_t first = (p.collapse ? ta : (ta | cls)) == 0 ? 0u : 1u;
+                // a tile starts from zero at its first MMA: the first class of the first K-tile (of
+                // this chunk of the K-slice), or, collapsed, the first K-tile (a collapsed tile
+                // belongs to one class only)
+                const uint32_t first = (p.collapse ? tac : (tac | cls)) == 0 ? 0u : 1u;
                 for (int u = mw; u < nunits; u += kMmaWarps) {
                     if (p.collapse && unit_cls[u] != cls) continue;
                     // A tap shifts the start by whole 128-byte rows. The swizzle is a function of
@@ -387,11 +424,14 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     __syncwarp();
 
     // ---------------------------------------------------------------- epilogue
-    if (warp >= 2 && warp < 6) {
-        bool ok = mbar_wait(&done_bar, 0, abort_flag);
+    const int nchunk_k = p.chunk_kt > 0 ? (kt_end - kt_begin + p.chunk_kt - 1) / p.chunk_kt : 1;
+    for (int kchunk = 0; warp >= 2 && warp < 6 && kchunk < nchunk_k; ++kchunk) {
+        bool ok = mbar_wait(&done_bar, kchunk & 1, abort_flag);
         if (!ok) flag_timeout(&abort_s, p.status, 0x300u);
         ok = __all_sync(0xffffffffu, ok);
-        if (ok) {
+        if (!ok) break;
+        const bool add_to = kchunk > 0;      // later chunks add to what the earlier ones stored
+        {
             tc_fence_after();
             const int quarter = warp & 3;            // the TMEM lanes this warp may read
             const int m = quarter * 32 + lane;       // accumulator row
@@ -417,8 +457,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                             if (m < p.CB) {
                                 float* q = dst + ((((long long)cob * p.ncib_total + cib0) * p.cu_total + cj0 + u) *
                                                       p.BN + cu * 32) * p.CB + m;
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) q[j * cstride] = __uint_as_float(buf[half][j]);
+                                put32(q, cstride, buf[half], add_to);
                             }
                             tap = -1; ci = 0;
                         } else if (p.pair_mode) {
@@ -431,13 +470,18 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                         }
                         if (tap >= 0) {
                             float* q = dst + ((long long)(co0 + cu * 32) * RS + tap) * p.Ci + ci;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) q[j * cstride] = __uint_as_float(buf[half][j]);
+                            put32(q, cstride, buf[half], add_to);
                         }
                         if (++cu == chunks_per_unit) { cu = 0; ++u; }
                     }
                 }
             }
+        }
+        if (kchunk + 1 < nchunk_k) {
+            // every tcgen05.ld of this warp has completed: the MMA warps may overwrite the tiles
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tfree_bar);
         }
     }
     tc_fence_before();
@@ -832,6 +876,13 @@ Tc2Geom build_geom2(const Dims& d, bool collapse) {
     if (splits < 1) splits = 1;
     if (splits > p.ktiles) splits = p.ktiles;
     p.splits = splits;
+    p.chunk_kt = 0;
+    if (d.max_chain > 0) {
+        // MMA instructions that add into one accumulator per K-tile: every class's, or, collapsed,
+        // those of the tile's own class
+        const int adds_per_ktile = (p.collapse ? 1 : p.ncls) * p.ksteps;
+        p.chunk_kt = d.max_chain / adds_per_ktile > 1 ? d.max_chain / adds_per_ktile : 1;
+    }
     g.smem_bytes = kSlotsA * p.a_slot_bytes + p.slotsB * p.b_slot_bytes + 1024;
     if (g.smem_bytes < 120 * 1024) g.smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
     g.ok = true;

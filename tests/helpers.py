@@ -111,12 +111,14 @@ def dw_to_oihw(dw: torch.Tensor, layout: str) -> np.ndarray:
     return a.transpose(0, 3, 1, 2) if layout == "nhwc" else a
 
 
-def run_wgrad(d: ac.ConvDesc, z, dy, dev="cuda:0", repeat=2):
+def run_wgrad(d: ac.ConvDesc, z, dy, dev="cuda:0", repeat=2, nbytes=None):
     """Runs the library `repeat` times (bitwise-equal results required) and
-    returns dW as float64 [Co,Ci,R,S]."""
+    returns dW as float64 [Co,Ci,R,S]. `nbytes`: workspace size to hand over
+    (default: what the fastest path asks for)."""
     zd = synth.to_layout(z, d.layout).to(dev)
     dyd = synth.to_layout(dy, d.layout).to(dev)
-    nbytes = ac.ac_workspace_bytes(d)
+    if nbytes is None:
+        nbytes = ac.ac_workspace_bytes(d)
     assert nbytes > 0
     outs = []
     for it in range(repeat):

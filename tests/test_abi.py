@@ -51,7 +51,14 @@ def test_workspace_bytes_is_host_only_and_rejects_bad_descriptors(ac):
 def test_workspace_grows_with_the_problem_not_unbounded(ac):
     small = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw")
     huge = ac.ConvDesc(256, 512, 512, 56, 56, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw")
-    assert ac.ac_workspace_bytes(small) < ac.ac_workspace_bytes(huge) < (1 << 30)
+    assert ac.ac_workspace_bytes_min(small) < ac.ac_workspace_bytes_min(huge) < (1 << 30)
+    # the fastest path for these fp32 NCHW problems stages six bf16 terms of each operand element
+    # (12 bytes each) and the kernel's dW on top of its partial sums: bounded by the problem, too
+    for d in (small, huge):
+        staged = 12 * (d.N * d.C_in * (d.H // 2) * (d.W // 2) + d.N * d.C_out * d.H * d.W) + 4 * d.C_out * d.C_in * 9
+        assert ac.ac_workspace_bytes_min(d) <= ac.ac_workspace_bytes(d) < (1 << 30) + staged + 4096
+    same = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
+    assert ac.ac_workspace_bytes_min(same) == ac.ac_workspace_bytes(same)
 
 
 def test_calls_validate_before_launching(ac):
@@ -135,8 +142,8 @@ def test_plan_info_respects_hardware_limits(ac):
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 28, 28, 3, 3, (2, 2), (1, 1), 1, "bf16", "nhwc"))
     assert i["tensor_core"] == 1
     # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
-    for d in (ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw"),
-              ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
+    for d in (ac.ConvDesc(8, 24, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw"),
+              ac.ConvDesc(8, 64, 40, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
               ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc"),
               ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (3, 3), (1, 1), 2, "bf16", "nhwc")):
         assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 0
@@ -146,7 +153,98 @@ def test_plan_info_respects_hardware_limits(ac):
     d16 = ac.ConvDesc(48, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
     i32, i16 = ac.ac_wgrad_plan_info(d32), ac.ac_wgrad_plan_info(d16)
     assert i32["tensor_core"] == 3 and i16["tensor_core"] == 2
-    assert {k: v for k, v in i32.items() if k != "tensor_core"} == {k: v for k, v in i16.items() if k != "tensor_core"}
+    # ... except that the K-slices are shorter (bounded accumulation chains), hence more of them
+    varies = ("tensor_core", "splits", "ctas")
+    assert {k: v for k, v in i32.items() if k not in varies} == {k: v for k, v in i16.items() if k not in varies}
+    assert i32["splits"] >= i16["splits"] and i32["ctas"] == i32["splits"] * i32["groups"]
     z6 = 48 * 64 * 16 * 16 * 2
     g6 = 48 * 64 * 32 * 32 * 2
-    assert ac.ac_workspace_bytes(d32) == ac.ac_workspace_bytes(d16) + z6 + g6
+    dw_bytes = 64 * 64 * 9 * 4
+    assert ac.ac_workspace_bytes(d32) == 256 + i32["splits"] * dw_bytes + z6 + g6
+    # NCHW inputs are transposed on the way: same kernel, plus room for its NHWC-ordered dW
+    for dt, mult in (("bf16", 1), ("f32", 6)):
+        dn = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, dt, "nchw")
+        info = ac.ac_wgrad_plan_info(dn)
+        assert info["tensor_core"] == 3
+        assert ac.ac_workspace_bytes(dn) == (256 + info["splits"] * dw_bytes + (z6 + g6) * mult // 6 + dw_bytes)
+
+
+def test_binding_fails_loudly_without_the_library(ac, monkeypatch):
+    monkeypatch.setattr(ac.api, "_lib", None)
+    monkeypatch.setattr(ac.api, "_LIB_PATH", "/nonexistent/libac.so")
+    with pytest.raises(ImportError):
+        ac.ac_workspace_bytes(ac.ConvDesc(1, 8, 8, 8, 8))
+
+
+def test_plan_info_respects_hardware_limits(ac):
+    """Host-side planning of the tensor-core path: shared memory, tensor memory
+    and pipeline depth stay inside what one SM has, for every benchmark layer."""
+    shapes = [
+        (64, 64, 64, 56, 56, 3, 3, 1, 1), (64, 128, 128, 28, 28, 3, 3, 1, 1),
+        (64, 256, 256, 14, 14, 3, 3, 1, 1), (64, 512, 512, 7, 7, 3, 3, 1, 1),
+        (64, 512, 512, 8, 8, 3, 3, 1, 1), (128, 256, 64, 56, 56, 1, 1, 1, 0),
+        (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
+        (256, 128, 128, 64, 64, 3, 3, 1, 1), (256, 1024, 2048, 14, 14, 1, 1, 2, 0),
+        (8, 64, 64, 30, 30, 7, 7, 2, 3), (2, 192, 320, 9, 40, 3, 3, 1, 1),
+    ]
+    for N, ci, co, H, W, R, S, st, pd in shapes:
+        for k in (1, 2, 4, 8):
+            d = ac.ConvDesc(N, ci, co, H, W, R, S, (st, st), (pd, pd), k, "bf16", "nhwc")
+            i = ac.ac_wgrad_plan_info(d)
+            assert i["tensor_core"] in (1, 2), d
+            assert 2 <= i["stages"] <= 8
+            assert i["smem_bytes"] <= 227 * 1024
+            assert i["tmem_columns"] in (32, 64, 128, 256, 512)
+            assert i["units_per_cta"] * i["block_n"] <= i["tmem_columns"]
+            assert i["k_tile"] % 16 == 0
+            if i["tensor_core"] == 1:
+                assert i["k_tile"] >= i["band_rows"] * i["row_pitch"]
+                assert i["row_pitch"] >= d.Wo
+            else:   # per class: (band_rows / c_h) class rows of row_pitch >= Wo / c_w positions
+                c_h, c_w = k // st, k // st
+                assert i["phases"] == c_h * c_w <= 64
+                assert i["k_tile"] >= (i["band_rows"] // c_h) * i["row_pitch"]
+                assert i["row_pitch"] >= -(-d.Wo // c_w)
+            assert 1 <= i["splits"] <= d.N * -(-d.Ho // i["band_rows"])
+            assert i["ctas"] == i["splits"] * i["groups"]
+            want = 256 + (i["splits"] * 4 * co * ci * R * S if i["splits"] > 1 else 0)
+            assert ac.ac_workspace_bytes(d) == want
+    # 64 input channels, 3x3, k = 2: the nine taps pair up into five accumulator tiles in one CTA
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 64, 64, 56, 56, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
+    assert (i["tensor_core"], i["units_per_cta"], i["groups"]) == (2, 5, 1)
+    # k = 8 at stride 1: 64 output classes, still the TMA-fed kernel
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(256, 128, 128, 64, 64, 3, 3, (1, 1), (1, 1), 8, "bf16", "nhwc"))
+    assert (i["tensor_core"], i["phases"]) == (2, 64)
+    # a map that k does not divide (partial pooling blocks) is still taken by the TMA-fed kernel
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 512, 512, 7, 7, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
+    assert i["tensor_core"] == 2
+    # a stride that does not divide k goes to the producer-fed tensor-core kernel
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 28, 28, 3, 3, (2, 2), (1, 1), 1, "bf16", "nhwc"))
+    assert i["tensor_core"] == 1
+    # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
+    for d in (ac.ConvDesc(8, 24, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw"),
+              ac.ConvDesc(8, 64, 40, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
+              ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc"),
+              ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (3, 3), (1, 1), 2, "bf16", "nhwc")):
+        assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 0
+    # fp32 NHWC goes to the tensor cores as six bf16 products: the same kernel on six times the
+    # images, with room for the split operands in the workspace
+    d32 = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nhwc")
+    d16 = ac.ConvDesc(48, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
+    i32, i16 = ac.ac_wgrad_plan_info(d32), ac.ac_wgrad_plan_info(d16)
+    assert i32["tensor_core"] == 3 and i16["tensor_core"] == 2
+    # ... except that the K-slices are shorter (bounded accumulation chains), hence more of them
+    varies = ("tensor_core", "splits", "ctas")
+    assert {k: v for k, v in i32.items() if k not in varies} == {k: v for k, v in i16.items() if k not in varies}
+    assert i32["splits"] >= i16["splits"] and i32["ctas"] == i32["splits"] * i32["groups"]
+    z6 = 48 * 64 * 16 * 16 * 2
+    g6 = 48 * 64 * 32 * 32 * 2
+    dw_bytes = 64 * 64 * 9 * 4
+    assert ac.ac_workspace_bytes(d32) == 256 + i32["splits"] * dw_bytes + z6 + g6
+    # NCHW inputs are transposed on the way: same kernel, plus room for its NHWC-ordered dW
+    for dt, mult in (("bf16", 1), ("f32", 6)):
+        dn = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, dt, "nchw")
+        di = ac.ConvDesc(8 * mult, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
+        assert ac.ac_wgrad_plan_info(dn)["tensor_core"] == 3
+        assert ac.ac_workspace_bytes(dn) == (ac.ac_workspace_bytes(di) + (z6 + g6) * mult // 6
+                                             + 64 * 64 * 9 * 4)

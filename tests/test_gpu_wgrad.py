@@ -95,6 +95,46 @@ def test_fp32_inputs_on_the_tensor_cores_full_size_sampled(N, Ci, Co, H, W, k):
     assert err <= 0.5 * TOL_DW["f32"], err
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("N,Ci,Co,H,W,R,stride,pad,k", [(64, 128, 128, 28, 28, 3, 1, 1, 2), (32, 64, 64, 56, 56, 3, 1, 1, 2),
+                                                         (16, 256, 64, 30, 30, 1, 1, 0, 2), (16, 128, 128, 27, 27, 3, 2, 1, 2),
+                                                         (8, 512, 512, 7, 7, 3, 1, 1, 2), (16, 64, 128, 24, 40, 3, 1, 1, 4)])
+def test_nchw_inputs_on_the_tensor_cores_full_size_sampled(N, Ci, Co, H, W, R, stride, pad, k, dtype):
+    """NCHW operands are transposed (and fp32 ones split) into the workspace; dW comes back in
+    NCHW order [Co][Ci][R][S]."""
+    import paper_2409_11902_b200 as ac
+    d = D(N, Ci, Co, H, W, R, R, stride, pad, k, dtype, "nchw")
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 3
+    err, _ = wgrad_error_sampled(d, n_samples=256)
+    assert err <= (0.5 * TOL_DW["f32"] if dtype == "f32" else TOL_DW["bf16"]), err
+
+
+def test_a_workspace_without_room_for_copies_takes_the_slower_path():
+    """With ac_workspace_bytes_min the same call runs on the operands as they are (fp32 FMA);
+    both results meet the bound, and the canary check shows neither writes past what it was given."""
+    import paper_2409_11902_b200 as ac
+    import oracle
+    from paper_2409_11902_b200 import synth
+    for dtype, layout in (("f32", "nhwc"), ("bf16", "nchw"), ("f32", "nchw")):
+        d = D(4, 64, 64, 20, 20, 3, 3, 1, 1, 2, dtype, layout)
+        lo, hi = ac.ac_workspace_bytes_min(d), ac.ac_workspace_bytes(d)
+        assert 256 <= lo < hi
+        z, dy = make_wgrad_inputs(d)
+        want = oracle.wgrad_compressed(synth.to_f64(z), synth.to_f64(dy), d.H, d.W, d.R, d.S, d.stride, d.pad, d.k)
+        for nbytes in (lo, hi - 256, hi):
+            got = run_wgrad(d, z, dy, nbytes=nbytes)
+            err = float(np.linalg.norm(got - want) / np.linalg.norm(want))
+            assert err <= TOL_DW[dtype], (dtype, layout, nbytes, err)
+        zd = synth.to_layout(z, layout).cuda()
+        dyd = synth.to_layout(dy, layout).cuda()
+        import torch
+        dw = torch.empty(d.dw_shape, dtype=torch.float32, device="cuda")
+        ws = torch.empty(hi, dtype=torch.uint8, device="cuda")
+        with pytest.raises(ac.AcError) as e:
+            ac.ac_conv2d_wgrad_compressed(d, zd, dyd, dw, ws, lo - 1)
+        assert e.value.status == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
+
+
 BOTTLENECK = [  # config 3: batch 128, bf16
     (128, 256, 64, 56, 56, 1, 1, 1, 0), (128, 64, 64, 56, 56, 3, 3, 1, 1),
     (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
