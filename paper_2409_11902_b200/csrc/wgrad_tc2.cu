@@ -117,13 +117,14 @@ __device__ __forceinline__ void flag_timeout(int* abort_s, uint32_t* status, uin
 // 32 accumulator columns of one row to memory, `stride` floats apart; `add_to`: added to what this
 // thread stored there before (all loads first, so that they overlap).
 __device__ __forceinline__ void put32(float* q, long long stride, const uint32_t* v, bool add_to) {
+    if (!add_to) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) q[j * stride] = __uint_as_float(v[j]);
+        return;
+    }
     float old[32];
 #pragma unroll
-    for (int j = 0; j < 32; ++j) old[j] = 0.f;
-    if (add_to) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) old[j] = q[j * stride];
-    }
+    for (int j = 0; j < 32; ++j) old[j] = q[j * stride];
 #pragma unroll
     for (int j = 0; j < 32; ++j) q[j * stride] = old[j] + __uint_as_float(v[j]);
 }
