@@ -158,6 +158,28 @@ ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc *desc, const void *z,
                                      size_t workspace_bytes, void *stream);
 
 /*
+ * The same weight gradient added to what dW holds (gradient accumulation over
+ * micro-batches): dW <- beta * dW + (the result of ac_conv2d_wgrad_compressed).
+ * The paper overwrites ("calculate the weight gradient normally", Section 4);
+ * this is the usual framework convenience on top. The new gradient is formed
+ * in the workspace by exactly the path ac_conv2d_wgrad_compressed would take
+ * with `workspace_bytes - 4*|dW|` bytes (rounded down to 256), then one pass
+ * combines it with dW, so the result is bitwise beta*dW + that gradient, in
+ * fp32. beta may be any finite value; beta == 0 still reads dW (NaNs in it
+ * propagate): call the plain entry point to overwrite.
+ *   workspace : at least ac_workspace_bytes_min(desc) rounded up to 256, plus
+ *               4*|dW| bytes;
+ *               ac_accumulate_workspace_bytes(desc) is the size for the
+ *               fastest path.
+ * Same return codes and status block as ac_conv2d_wgrad_compressed.
+ */
+size_t ac_accumulate_workspace_bytes(const ac_conv_desc *desc);
+ac_status ac_conv2d_wgrad_compressed_accumulate(const ac_conv_desc *desc, const void *z,
+                                                const void *dy, float beta, float *dw,
+                                                void *workspace, size_t workspace_bytes,
+                                                void *stream);
+
+/*
  * Reads back the status block a previous ac_conv2d_wgrad_compressed call left
  * in `workspace`: synchronises `stream`, then returns AC_OK, or AC_ERR_TIMEOUT
  * if a bounded wait inside a kernel gave up (dW is then not valid), or

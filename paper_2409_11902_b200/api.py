@@ -70,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.ac_compress_relu_mask.argtypes = [dp, vp, vp, vp, vp]
         L.ac_conv2d_wgrad_compressed.restype = ctypes.c_int
         L.ac_conv2d_wgrad_compressed.argtypes = [dp, vp, vp, vp, vp, sz, vp]
+        L.ac_accumulate_workspace_bytes.restype = sz
+        L.ac_accumulate_workspace_bytes.argtypes = [dp]
+        L.ac_conv2d_wgrad_compressed_accumulate.restype = ctypes.c_int
+        L.ac_conv2d_wgrad_compressed_accumulate.argtypes = [dp, vp, vp, ctypes.c_float, vp, vp, sz, vp]
         L.ac_workspace_status.restype = ctypes.c_int
         L.ac_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
         L.ac_host_step_arena_bytes.restype = sz
@@ -196,6 +200,22 @@ def ac_conv2d_wgrad_compressed(desc: ConvDesc, z, dy, dw, workspace, workspace_b
                                           _ptr(workspace), workspace_bytes, _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_conv2d_wgrad_compressed")
+
+
+def ac_accumulate_workspace_bytes(desc: ConvDesc) -> int:
+    c = desc.c()
+    return int(lib().ac_accumulate_workspace_bytes(ctypes.byref(c)))
+
+
+def ac_conv2d_wgrad_compressed_accumulate(desc: ConvDesc, z, dy, beta, dw, workspace, workspace_bytes=None,
+                                          stream=None) -> None:
+    c = desc.c()
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    st = lib().ac_conv2d_wgrad_compressed_accumulate(ctypes.byref(c), _ptr(z), _ptr(dy), float(beta), _ptr(dw),
+                                                     _ptr(workspace), workspace_bytes, _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_conv2d_wgrad_compressed_accumulate")
 
 
 def ac_workspace_status(workspace, stream=None):

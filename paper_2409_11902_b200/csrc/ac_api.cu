@@ -148,6 +148,32 @@ ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, co
     return launch_wgrad_simt(d, p, z, dy, dw, workspace, s);
 }
 
+size_t ac_accumulate_workspace_bytes(const ac_conv_desc* desc) {
+    Dims d;
+    if (make_dims(desc, true, &d) != AC_OK) return 0;
+    return ((plan_wgrad(d).bytes + 255) & ~(size_t)255) + (size_t)d.dw_elems() * 4;
+}
+
+ac_status ac_conv2d_wgrad_compressed_accumulate(const ac_conv_desc* desc, const void* z, const void* dy,
+                                                float beta, float* dw, void* workspace,
+                                                size_t workspace_bytes, void* stream) {
+    Dims d;
+    ac_status st = make_dims(desc, true, &d);
+    if (st != AC_OK) return st;
+    if (!dw || !workspace) return AC_ERR_INVALID_ARG;
+    if (!aligned16(dw)) return AC_ERR_MISALIGNED;
+    if (!(beta == beta) || beta - beta != 0.f) return AC_ERR_INVALID_ARG;   // NaN or infinite
+    const size_t dw_bytes = (size_t)d.dw_elems() * 4;
+    if (workspace_bytes < dw_bytes + 256) return AC_ERR_WORKSPACE_TOO_SMALL;
+    // the gradient's own scratch in front (so that the status block stays where ac_workspace_status
+    // looks for it), the new gradient behind it
+    const size_t inner = (workspace_bytes - dw_bytes) & ~(size_t)255;
+    float* g = reinterpret_cast<float*>(static_cast<char*>(workspace) + inner);
+    st = ac_conv2d_wgrad_compressed(desc, z, dy, g, workspace, inner, stream);
+    if (st != AC_OK) return st;
+    return launch_axpby(g, beta, dw, d.dw_elems(), static_cast<cudaStream_t>(stream));
+}
+
 ac_status ac_workspace_status(const void* workspace, void* stream, uint32_t* detail) {
     if (!workspace) return AC_ERR_INVALID_ARG;
     uint32_t word[2] = {0, 0};

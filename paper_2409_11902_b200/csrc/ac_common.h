@@ -84,6 +84,7 @@ size_t tc2_collapsed_workspace_bytes(const Dims& d, int* tiles_collapsed, int* t
 ac_status launch_wgrad_tc2_collapsed(const Dims& d, const void* z, const void* dy, float* dw,
                                      void* workspace, cudaStream_t stream);
 ac_status launch_bounded_wait_selftest(void* workspace, long long limit_cycles, cudaStream_t stream);
+ac_status launch_axpby(const float* g, float beta, float* dw, long long elems, cudaStream_t stream);
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
                                cudaStream_t stream);
 

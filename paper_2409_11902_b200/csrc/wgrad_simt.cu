@@ -208,6 +208,20 @@ void launch_reduce4(const float* partials, int splits, long long e4, float* dw, 
 
 }  // namespace
 
+namespace {
+__global__ void __launch_bounds__(256) axpby_kernel(const float* __restrict__ g, float beta, float* dw, long long n) {
+    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (i < n) dw[i] = __fmaf_rn(beta, dw[i], g[i]);
+}
+}  // namespace
+
+// dw <- beta * dw + g (one rounding per element)
+ac_status launch_axpby(const float* g, float beta, float* dw, long long elems, cudaStream_t stream) {
+    axpby_kernel<<<(unsigned)((elems + 255) / 256), 256, 0, stream>>>(g, beta, dw, elems);
+    AC_CUDA_TRY(cudaGetLastError());
+    return AC_OK;
+}
+
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
                                cudaStream_t stream) {
     if (elems % 4 == 0) {

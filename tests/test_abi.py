@@ -84,6 +84,15 @@ def test_calls_validate_before_launching(ac):
     bad = ac.ConvDesc(2, 8, 8, 8, 8, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw").c()
     bad.dtype = 7
     assert L.ac_compress(ctypes.byref(bad), A, A, None, None) == ac.api.AC_ERR_INVALID_ARG
+    acc = L.ac_conv2d_wgrad_compressed_accumulate
+    assert acc(ref, A, A, 1.0, None, A, 1 << 30, None) == ac.api.AC_ERR_INVALID_ARG
+    assert acc(ref, A, A, 1.0, A + 4, A, 1 << 30, None) == ac.api.AC_ERR_MISALIGNED
+    assert acc(ref, A, A, float("nan"), A, A, 1 << 30, None) == ac.api.AC_ERR_INVALID_ARG
+    assert acc(ref, A, A, float("inf"), A, A, 1 << 30, None) == ac.api.AC_ERR_INVALID_ARG
+    assert acc(ref, A, A, 1.0, A, A, 8 * 8 * 9 * 4 + 255, None) == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
+    assert acc(ref, A, None, 1.0, A, A, 1 << 30, None) == ac.api.AC_ERR_INVALID_ARG
+    good = ac.ConvDesc(2, 8, 8, 8, 8, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw")
+    assert ac.ac_accumulate_workspace_bytes(good) >= ac.ac_workspace_bytes(good) + 8 * 8 * 9 * 4
     assert L.ac_backward_step_host(ref, A, A, A, None, A + 16, 1 << 30, None) == ac.api.AC_ERR_MISALIGNED
     assert L.ac_backward_step_host(ref, A, A, A, None, A, 16, None) == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
     assert L.ac_workspace_status(None, None, None) == ac.api.AC_ERR_INVALID_ARG

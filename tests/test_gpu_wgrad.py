@@ -135,6 +135,39 @@ def test_a_workspace_without_room_for_copies_takes_the_slower_path():
         assert e.value.status == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
 
 
+@pytest.mark.parametrize("dtype,layout", [("bf16", "nhwc"), ("f32", "nchw"), ("f32", "nhwc"), ("bf16", "nchw")])
+def test_accumulate_adds_to_what_dw_holds(dtype, layout):
+    """dW <- beta * dW + gradient: with beta = 1 on zeros it is the plain call bit for bit; with
+    beta = 0.5 on a random dW it is the fused multiply-add of the two; any workspace from the
+    minimum up is taken."""
+    import torch
+    import paper_2409_11902_b200 as ac
+    from paper_2409_11902_b200 import synth
+    d = D(4, 64, 64, 20, 20, 3, 3, 1, 1, 2, dtype, layout)
+    z, dy = make_wgrad_inputs(d)
+    zd = synth.to_layout(z, layout).cuda()
+    dyd = synth.to_layout(dy, layout).cuda()
+    dw_bytes = 64 * 64 * 9 * 4
+    for nbytes, plain_bytes in ((ac.ac_accumulate_workspace_bytes(d), ac.ac_workspace_bytes(d)),
+                                (ac.ac_workspace_bytes_min(d) + dw_bytes + 256, ac.ac_workspace_bytes_min(d))):
+        plain = torch.empty(d.dw_shape, dtype=torch.float32, device="cuda")
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        ac.ac_conv2d_wgrad_compressed(d, zd, dyd, plain, ws, plain_bytes)
+        dw = torch.zeros_like(plain)
+        ac.ac_conv2d_wgrad_compressed_accumulate(d, zd, dyd, 1.0, dw, ws)
+        assert ac.ac_workspace_status(ws)[0] == 0
+        assert torch.equal(dw, plain)
+        g = torch.Generator(device="cuda").manual_seed(5)
+        old = torch.randn(d.dw_shape, generator=g, device="cuda") * plain.abs().mean()
+        dw = old.clone()
+        ac.ac_conv2d_wgrad_compressed_accumulate(d, zd, dyd, 0.5, dw, ws)
+        want = (0.5 * old.double() + plain.double())
+        assert float((dw.double() - want).abs().max()) <= 1.2e-7 * float(want.abs().max())
+        with pytest.raises(ac.AcError) as e:
+            ac.ac_conv2d_wgrad_compressed_accumulate(d, zd, dyd, 1.0, dw, ws, ac.ac_workspace_bytes_min(d) + dw_bytes - 1)
+        assert e.value.status == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
+
+
 BOTTLENECK = [  # config 3: batch 128, bf16
     (128, 256, 64, 56, 56, 1, 1, 1, 0), (128, 64, 64, 56, 56, 3, 3, 1, 1),
     (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
