@@ -242,8 +242,11 @@ ac_status ac_conv2d_wgrad_compressed_static(const ac_conv_desc *desc, const void
  * reports and tests). Returns AC_ERR_INVALID_ARG for an invalid descriptor.
  */
 typedef struct {
-    int32_t tensor_core;     /* 3: fp32 inputs split into bf16 terms, then as 2 with six times the
-                                images (the other fields describe that launch), 2: TMA-fed tcgen05
+    int32_t tensor_core;     /* 4: as 3, but as two launches whose results are added: the five small
+                                partial products (five times the images; described by the other
+                                fields), then the leading one, 3: fp32 and/or NCHW inputs staged
+                                as bf16 NHWC terms in the workspace (fp32: six partial products =
+                                six times the images), then as 2, 2: TMA-fed tcgen05
                                 kernel, 1: tcgen05 kernel with inflating producer warps,
                                 0: fp32-ALU kernel */
     int32_t splits;          /* K-slices summed by the split-K reduction */

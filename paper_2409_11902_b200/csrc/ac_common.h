@@ -51,7 +51,7 @@ struct WgradPlan {
     int tc_ktiles;   // K-tiles in the whole problem
     int tc_stages;   // shared-memory pipeline depth
     // staged path: where the staged operands and (NCHW) the kernel's dW sit in the workspace
-    size_t st_off_z, st_off_dy, st_off_dw;
+    size_t st_off_z, st_off_dy, st_off_dw, st_off_small;
     size_t bytes;    // workspace bytes including the status block
 };
 
@@ -73,7 +73,8 @@ bool tc2_supported(const Dims& d, double* k_eff);
 void plan_tc2(const Dims& d, WgradPlan* p);
 void tc2_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
-                           float* dw, void* workspace, cudaStream_t stream);
+                           float* dw, void* workspace, cudaStream_t stream, bool keep_status = false);
+int tc2_chain_length(const Dims& d);
 // fp32 and/or NCHW inputs staged for the TMA-fed kernel (wgrad_staged.cu)
 bool staged_supported(const Dims& d);
 void plan_staged(const Dims& d, WgradPlan* p);

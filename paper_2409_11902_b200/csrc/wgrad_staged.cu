@@ -11,9 +11,12 @@
 //    all accumulated in fp32. A weight gradient is a sum over images, so the six products are simply
 //    six times as many images for the bf16 kernel:
 //
-//        Z'  = [ Zh | Zh | Zm | Zh | Zl | Zm ]        dY' = [ Gh | Gm | Gh | Gl | Gh | Gm ]
+//        Z'  = [ Zh | Zm | Zh | Zl | Zm | Zh ]        dY' = [ Gm | Gh | Gl | Gh | Gm | Gh ]
 //
-//    (each block N images, bf16), and the kernel runs unchanged with N' = 6 N. Against the fp64
+//    (each block N images, bf16; the leading product Zh*Gh last), and the kernel runs unchanged with
+//    N' = 6 N. When the accumulation chains of that launch would need to be cut often (see
+//    kMaxChainF32), the five small products (5 N images, sums 2^-8 of the result and less, no bound
+//    needed) and the leading one (N images) are run as two launches and added. Against the fp64
 //    definition the relative Frobenius error is 7e-7 .. 2e-6 (fp32-ALU path: 3e-7 .. 5e-7, at a
 //    fifth to a tenth of the speed).
 //
@@ -41,8 +44,8 @@ __device__ __forceinline__ void split3(float x, float& h, float& m, float& l) {
 // Which of (h, m, l) goes to block b of the staged tensor: ROLE 0 is Z', ROLE 1 is dY'.
 template <int ROLE>
 __device__ __forceinline__ int term_of_block(int b) {
-    // Z': h h m h l m      dY': h m h l h m
-    return ROLE == 0 ? ((0x120100 >> (4 * b)) & 3) : ((0x102010 >> (4 * b)) & 3);
+    // Z': h m h l m h      dY': m h l h m h
+    return ROLE == 0 ? ((0x012010 >> (4 * b)) & 3) : ((0x010201 >> (4 * b)) & 3);
 }
 
 // fp32 NHWC -> six bf16 blocks. One thread splits 8 consecutive values and stores three 16-byte
@@ -131,8 +134,13 @@ inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 //     128       1.6e-6 / 151 us  (1.3e-6 / 332 us)
 constexpr int kMaxChainF32 = 128;
 
-// The bf16 NHWC problem the staged operands amount to.
-bool inner_problem(const Dims& d, Dims* in) {
+// The bf16 NHWC problem(s) the staged operands amount to: `a` is the first launch; `b.N > 0` means
+// a second launch on the last block alone (the leading product), whose result is added to the first's.
+struct Inner {
+    Dims a, b;
+};
+
+bool inner_problem(const Dims& d, Inner* out) {
     const bool split = d.dtype == AC_F32, transpose = d.layout == AC_NCHW;
     if (!split && !transpose) return false;                 // the kernel reads these itself
     if (transpose) {
@@ -143,15 +151,35 @@ bool inner_problem(const Dims& d, Dims* in) {
     }
     const long long n_in = (long long)d.N * (split ? 6 : 1);
     if (n_in >= (1ll << 31)) return false;
-    *in = d;
-    in->N = (int)n_in;
-    in->dtype = AC_BF16;
-    in->layout = AC_NHWC;
-    in->elt = 2;
-    if (split) in->max_chain = kMaxChainF32;
+    Dims in = d;
+    in.N = (int)n_in;
+    in.dtype = AC_BF16;
+    in.layout = AC_NHWC;
+    in.elt = 2;
     const long long lim = 1ll << 40;
-    if (in->z_elems() >= lim || in->dy_elems() >= lim) return false;
-    return tc2_supported(*in, nullptr);
+    if (in.z_elems() >= lim || in.dy_elems() >= lim) return false;
+    out->a = in;
+    out->b = in;
+    out->b.N = 0;
+    if (!split) return tc2_supported(in, nullptr);
+    // one launch with bounded chains, or two: each cut of the chains costs a read-add-store of the
+    // accumulators (about 6 us), a second launch about 20 us of fixed work
+    Dims one = in, small = in, lead = in;
+    one.max_chain = kMaxChainF32;
+    small.N = d.N * 5;
+    lead.N = d.N;
+    lead.max_chain = kMaxChainF32;
+    if (!tc2_supported(one, nullptr)) return false;
+    out->a = one;
+    if (tc2_supported(small, nullptr) && tc2_supported(lead, nullptr)) {
+        const int cuts_one = (tc2_chain_length(one) + kMaxChainF32 - 1) / kMaxChainF32 - 1;
+        const int cuts_lead = (tc2_chain_length(lead) + kMaxChainF32 - 1) / kMaxChainF32 - 1;
+        if (6 * cuts_one > 20 + 6 * cuts_lead) {
+            out->a = small;
+            out->b = lead;
+        }
+    }
+    return true;
 }
 
 template <typename TIN, bool SPLIT>
@@ -169,35 +197,42 @@ ac_status stage_nchw(const TIN* z, const TIN* dy, void* z_st, void* dy_st, const
 }  // namespace
 
 bool staged_supported(const Dims& d) {
-    Dims in;
+    Inner in;
     return inner_problem(d, &in);
 }
 
 void plan_staged(const Dims& d, WgradPlan* pl) {
-    Dims in;
+    Inner in;
     inner_problem(d, &in);
-    plan_tc2(in, pl);
+    plan_tc2(in.a, pl);
+    if (in.b.N > 0) {
+        WgradPlan pb{};
+        plan_tc2(in.b, &pb);
+        if (pb.bytes > pl->bytes) pl->bytes = pb.bytes;     // the launches use the partial sums' room in turn
+    }
+    const long long blocks = d.dtype == AC_F32 ? 6 : 1;
     pl->path = PATH_STAGED;
     pl->st_off_z = up256(pl->bytes);
-    pl->st_off_dy = pl->st_off_z + up256((size_t)in.z_elems() * 2);
-    pl->st_off_dw = pl->st_off_dy + up256((size_t)in.dy_elems() * 2);
-    pl->bytes = pl->st_off_dw + (d.layout == AC_NCHW ? up256((size_t)d.dw_elems() * 4) : 0);
+    pl->st_off_dy = pl->st_off_z + up256((size_t)(d.z_elems() * blocks) * 2);
+    pl->st_off_dw = pl->st_off_dy + up256((size_t)(d.dy_elems() * blocks) * 2);
+    pl->st_off_small = pl->st_off_dw + (d.layout == AC_NCHW ? up256((size_t)d.dw_elems() * 4) : 0);
+    pl->bytes = pl->st_off_small + (in.b.N > 0 ? up256((size_t)d.dw_elems() * 4) : 0);
 }
 
 void staged_plan_info(const Dims& d, ac_plan_info* info) {
-    Dims in;
+    Inner in;
     inner_problem(d, &in);
-    tc2_plan_info(in, info);
-    info->tensor_core = 3;
+    tc2_plan_info(in.a, info);
+    info->tensor_core = in.b.N > 0 ? 4 : 3;
 }
 
 ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z, const void* dy,
                               float* dw, void* workspace, cudaStream_t stream) {
-    Dims in;
+    Inner in;
     if (!inner_problem(d, &in)) return AC_ERR_UNSUPPORTED;
     char* ws = static_cast<char*>(workspace);
-    void* z_st = ws + pl.st_off_z;
-    void* dy_st = ws + pl.st_off_dy;
+    char* z_st = ws + pl.st_off_z;
+    char* dy_st = ws + pl.st_off_dy;
     ac_status st = AC_OK;
     if (d.layout == AC_NCHW) {
         if (d.dtype == AC_F32)
@@ -210,17 +245,30 @@ ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z,
         const long long nz8 = d.z_elems() / 8, ng8 = d.dy_elems() / 8;
         if ((nz8 + 255) / 256 >= (1ll << 31) || (ng8 + 255) / 256 >= (1ll << 31)) return AC_ERR_UNSUPPORTED;
         split3_kernel<0><<<(unsigned)((nz8 + 255) / 256), 256, 0, stream>>>(
-            static_cast<const float4*>(z), static_cast<uint4*>(z_st), nz8);
+            reinterpret_cast<const float4*>(z), reinterpret_cast<uint4*>(z_st), nz8);
         split3_kernel<1><<<(unsigned)((ng8 + 255) / 256), 256, 0, stream>>>(
-            static_cast<const float4*>(dy), static_cast<uint4*>(dy_st), ng8);
+            reinterpret_cast<const float4*>(dy), reinterpret_cast<uint4*>(dy_st), ng8);
         AC_CUDA_TRY(cudaGetLastError());
     }
-    if (d.layout == AC_NHWC) return launch_wgrad_tc2(in, pl, z_st, dy_st, dw, workspace, stream);
-    float* dw_st = reinterpret_cast<float*>(ws + pl.st_off_dw);
-    st = launch_wgrad_tc2(in, pl, z_st, dy_st, dw_st, workspace, stream);
-    if (st != AC_OK) return st;
+    // where the kernel's [C_out][R][S][C_in] result goes: the caller's dW, or the workspace if it
+    // still has to be permuted
+    float* out_nhwc = d.layout == AC_NHWC ? dw : reinterpret_cast<float*>(ws + pl.st_off_dw);
+    if (in.b.N == 0) {
+        st = launch_wgrad_tc2(in.a, pl, z_st, dy_st, out_nhwc, workspace, stream);
+        if (st != AC_OK) return st;
+    } else {
+        float* small = reinterpret_cast<float*>(ws + pl.st_off_small);
+        st = launch_wgrad_tc2(in.a, pl, z_st, dy_st, small, workspace, stream);
+        if (st != AC_OK) return st;
+        st = launch_wgrad_tc2(in.b, pl, z_st + (size_t)d.z_elems() * 5 * 2, dy_st + (size_t)d.dy_elems() * 5 * 2,
+                              out_nhwc, workspace, stream, /*keep_status=*/true);
+        if (st != AC_OK) return st;
+        st = launch_axpby(small, 1.0f, out_nhwc, d.dw_elems(), stream);     // leading product + the rest
+        if (st != AC_OK) return st;
+    }
+    if (d.layout == AC_NHWC) return AC_OK;
     const long long total = d.dw_elems();
-    permute_dw_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(dw_st, dw, d.Ci, d.R * d.S, total);
+    permute_dw_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(out_nhwc, dw, d.Ci, d.R * d.S, total);
     AC_CUDA_TRY(cudaGetLastError());
     return AC_OK;
 }

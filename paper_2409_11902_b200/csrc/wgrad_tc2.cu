@@ -55,6 +55,7 @@ struct Tc2Params {
     int strided_map;
     float* out;
     uint32_t* status;
+    int keep_status;   // 1: a launch earlier in the same call owns the status block; do not reset it
     int Ci, Co, R, S, sh, sw, ph, pw, k;
     int c_h, c_w, ncls;
     int umin, vmin;
@@ -178,7 +179,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
 
     // The status block starts clean: CTA 0 resets it here, long before any wait of this launch
     // can run out (a wait gives up only after 2^32 cycles).
-    if (blockIdx.x == 0 && tid == 0) { p.status[0] = 0u; p.status[1] = 0u; }
+    if (blockIdx.x == 0 && tid == 0 && !p.keep_status) { p.status[0] = 0u; p.status[1] = 0u; }
 
     // ---------------------------------------------------------------- TMA producer
     // Warp 0 issues every copy. The stream of copies is: for each K-tile, the Z halo
@@ -978,10 +979,11 @@ void tc2_plan_info(const Dims& d, ac_plan_info* info) {
 }
 
 static ac_status launch_tc2_any(const Dims& d, bool collapse, const void* z, const void* dy, float* dw,
-                                void* workspace, cudaStream_t stream) {
+                                void* workspace, cudaStream_t stream, bool keep_status = false) {
     Tc2Geom g = make_geom2(d, collapse);
     if (!g.ok) return AC_ERR_UNSUPPORTED;
     Tc2Params& p = g.p;
+    p.keep_status = keep_status ? 1 : 0;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return AC_ERR_CUDA;
     for (int var = 0; var < 4; ++var) {
@@ -1060,9 +1062,16 @@ static ac_status launch_tc2_any(const Dims& d, bool collapse, const void* z, con
 }
 
 ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& pl, const void* z, const void* dy,
-                           float* dw, void* workspace, cudaStream_t stream) {
+                           float* dw, void* workspace, cudaStream_t stream, bool keep_status) {
     (void)pl;
-    return launch_tc2_any(d, false, z, dy, dw, workspace, stream);
+    return launch_tc2_any(d, false, z, dy, dw, workspace, stream, keep_status);
+}
+
+// MMA instructions that add into one accumulator over a CTA's whole K-slice
+int tc2_chain_length(const Dims& d) {
+    const Tc2Geom g = make_geom2(d);
+    if (!g.ok) return 0;
+    return (g.p.ktiles + g.p.splits - 1) / g.p.splits * g.p.ncls * g.p.ksteps;
 }
 
 // Collapsed form: same dW, fewer MMAs (see Tc2Params::collapse). 0 bytes / AC_ERR_UNSUPPORTED when the

@@ -90,7 +90,7 @@ def test_fp32_inputs_on_the_tensor_cores_full_size_sampled(N, Ci, Co, H, W, k):
     at least a factor of two to spare, at sizes where each entry sums 10^4 .. 10^5 products."""
     import paper_2409_11902_b200 as ac
     d = D(N, Ci, Co, H, W, 3, 3, 1, 1, k, "f32", "nhwc")
-    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 3
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] in (3, 4)
     err, _ = wgrad_error_sampled(d, n_samples=256)
     assert err <= 0.5 * TOL_DW["f32"], err
 
@@ -104,7 +104,7 @@ def test_nchw_inputs_on_the_tensor_cores_full_size_sampled(N, Ci, Co, H, W, R, s
     NCHW order [Co][Ci][R][S]."""
     import paper_2409_11902_b200 as ac
     d = D(N, Ci, Co, H, W, R, R, stride, pad, k, dtype, "nchw")
-    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 3
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] in (3, 4)
     err, _ = wgrad_error_sampled(d, n_samples=256)
     assert err <= (0.5 * TOL_DW["f32"] if dtype == "f32" else TOL_DW["bf16"]), err
 
