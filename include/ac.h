@@ -180,6 +180,18 @@ ac_status ac_conv2d_wgrad_compressed_accumulate(const ac_conv_desc *desc, const 
                                                 void *stream);
 
 /*
+ * Profiling aid (not part of the paper's method). While a pair of CUDA events
+ * (cudaEvent_t, created with timing enabled) is set for the calling host thread,
+ * every weight-gradient call made from that thread records `before` and
+ * `after` on its stream immediately around the main weight-gradient kernel
+ * alone: not the staging passes, not the split-K reduction (with two main
+ * launches in one call the events end up around the last). Under stream
+ * capture the records become external event-record nodes of the graph.
+ * Passing NULL for either clears the pair. The events stay the caller's.
+ */
+ac_status ac_set_kernel_timing_events(void *before, void *after);
+
+/*
  * Reads back the status block a previous ac_conv2d_wgrad_compressed call left
  * in `workspace`: synchronises `stream`, then returns AC_OK, or AC_ERR_TIMEOUT
  * if a bounded wait inside a kernel gave up (dW is then not valid), or

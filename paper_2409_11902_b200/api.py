@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.ac_accumulate_workspace_bytes.argtypes = [dp]
         L.ac_conv2d_wgrad_compressed_accumulate.restype = ctypes.c_int
         L.ac_conv2d_wgrad_compressed_accumulate.argtypes = [dp, vp, vp, ctypes.c_float, vp, vp, sz, vp]
+        L.ac_set_kernel_timing_events.restype = ctypes.c_int
+        L.ac_set_kernel_timing_events.argtypes = [vp, vp]
         L.ac_workspace_status.restype = ctypes.c_int
         L.ac_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
         L.ac_host_step_arena_bytes.restype = sz
@@ -216,6 +218,18 @@ def ac_conv2d_wgrad_compressed_accumulate(desc: ConvDesc, z, dy, beta, dw, works
                                                      _ptr(workspace), workspace_bytes, _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_conv2d_wgrad_compressed_accumulate")
+
+
+def ac_set_kernel_timing_events(before=None, after=None) -> None:
+    """`before`, `after`: torch.cuda.Event objects (already recorded once or created eagerly, so that
+    their handles exist) or raw cudaEvent_t integers; None clears."""
+    def raw(e):
+        if e is None:
+            return None
+        return int(getattr(e, "cuda_event", e))
+    st = lib().ac_set_kernel_timing_events(raw(before), raw(after))
+    if st != AC_OK:
+        raise AcError(st, "ac_set_kernel_timing_events")
 
 
 def ac_workspace_status(workspace, stream=None):

@@ -59,6 +59,19 @@ WgradPlan plan_wgrad_simt(const Dims& d) {
     return p;
 }
 
+namespace {
+thread_local cudaEvent_t g_hook_events[2] = {nullptr, nullptr};
+}
+
+void record_timing_hook(int which, cudaStream_t stream) {
+    cudaEvent_t ev = g_hook_events[which];
+    if (!ev) return;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess) return;
+    cudaEventRecordWithFlags(ev, stream,
+                             cs == cudaStreamCaptureStatusActive ? cudaEventRecordExternal : cudaEventRecordDefault);
+}
+
 // The plan for a caller whose workspace has no room for staged operand copies.
 WgradPlan plan_wgrad_unstaged(const Dims& d) {
     if (tc_supported(d)) {
@@ -172,6 +185,13 @@ ac_status ac_conv2d_wgrad_compressed_accumulate(const ac_conv_desc* desc, const 
     st = ac_conv2d_wgrad_compressed(desc, z, dy, g, workspace, inner, stream);
     if (st != AC_OK) return st;
     return launch_axpby(g, beta, dw, d.dw_elems(), static_cast<cudaStream_t>(stream));
+}
+
+ac_status ac_set_kernel_timing_events(void* before, void* after) {
+    const bool on = before && after;
+    g_hook_events[0] = on ? static_cast<cudaEvent_t>(before) : nullptr;
+    g_hook_events[1] = on ? static_cast<cudaEvent_t>(after) : nullptr;
+    return AC_OK;
 }
 
 ac_status ac_workspace_status(const void* workspace, void* stream, uint32_t* detail) {

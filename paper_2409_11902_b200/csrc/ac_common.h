@@ -89,6 +89,9 @@ ac_status launch_axpby(const float* g, float beta, float* dw, long long elems, c
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
                                cudaStream_t stream);
 
+// Profiling hook (ac_set_kernel_timing_events): which = 0 before, 1 after the main kernel.
+void record_timing_hook(int which, cudaStream_t stream);
+
 // Raises a kernel's dynamic shared-memory limit once per device (the attribute is per device).
 template <typename Kernel>
 inline ac_status ensure_smem_limit(Kernel kernel, int bytes, bool (&done)[64]) {

@@ -261,11 +261,13 @@ ac_status launch_wgrad_simt(const Dims& d, const WgradPlan& pl, const void* z, c
     float* out = pl.splits > 1 ? partials : dw;
     dim3 grid((p.J + BN - 1) / BN, (d.Co + BM - 1) / BM, pl.splits);
     if (grid.y > 65535u || grid.z > 65535u) return AC_ERR_UNSUPPORTED;
+    record_timing_hook(0, stream);
     if (d.dtype == AC_F32)
         wgrad_simt_kernel<float><<<grid, 256, 0, stream>>>((const float*)z, (const float*)dy, out, p);
     else
         wgrad_simt_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
             (const __nv_bfloat16*)z, (const __nv_bfloat16*)dy, out, p);
+    record_timing_hook(1, stream);
     AC_CUDA_TRY(cudaGetLastError());
     if (pl.splits > 1) return launch_splitk_reduce(partials, pl.splits, p.dw_elems, dw, stream);
     return AC_OK;

@@ -443,7 +443,9 @@ ac_status launch_wgrad_tc(const Dims& d, const WgradPlan& pl, const void* z, con
         const ac_status st_ = ensure_smem_limit(wgrad_tc_kernel, (int)kSmemBudget, attr_done);
         if (st_ != AC_OK) return st_;
     }
+    record_timing_hook(0, stream);
     wgrad_tc_kernel<<<p.groups * p.splits, kThreads, g.smem_bytes, stream>>>(p);
+    record_timing_hook(1, stream);
     AC_CUDA_TRY(cudaGetLastError());
     if (p.splits > 1) return launch_splitk_reduce(partials, p.splits, p.dw_elems, dw, stream);
     (void)pl;

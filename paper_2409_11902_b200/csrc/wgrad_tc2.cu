@@ -1036,7 +1036,9 @@ static ac_status launch_tc2_any(const Dims& d, bool collapse, const void* z, con
         const ac_status st_ = ensure_smem_limit(wgrad_tc2_kernel, (int)(kSmemBudget2 + 1024), attr_done);
         if (st_ != AC_OK) return st_;
     }
+    record_timing_hook(0, stream);
     wgrad_tc2_kernel<<<p.groups * p.splits, kThreads2, g.smem_bytes, stream>>>(p);
+    record_timing_hook(1, stream);
     AC_CUDA_TRY(cudaGetLastError());
     if (p.collapse) {
         CollapseReduceParams q;
