@@ -89,6 +89,36 @@ ac_status launch_axpby(const float* g, float beta, float* dw, long long elems, c
 ac_status launch_splitk_reduce(const float* partials, int splits, long long elems, float* dw,
                                cudaStream_t stream);
 
+// Programmatic dependent launch. A kernel launched with launch_after() may start while the kernel
+// before it in the stream is still running, provided that kernel has called
+// pdl_launch_dependents() in every CTA; whatever it does before pdl_wait() (barrier set-up, TMEM
+// allocation, clearing shared memory) then overlaps the predecessor's tail. pdl_wait() returns once
+// the predecessor has completed and its writes are visible; every thread calls it before its first
+// access to global memory. With a predecessor that never signals, the launch behaves like an
+// ordinary one and pdl_wait() returns at once.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Profiling hook (ac_set_kernel_timing_events): which = 0 before, 1 after the main kernel.
 void record_timing_hook(int which, cudaStream_t stream);
 

@@ -129,6 +129,7 @@ template <typename T, int K, int MODE>   // MODE 0: pool only, 1: also store max
 __global__ void __launch_bounds__(256)
 compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int CV,
                   int k, int Hp, int Wp) {
+    pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
     constexpr bool RELU = MODE != 0;
     constexpr int VW = VecTraits<T>::VW;
     const unsigned item = blockIdx.x * 256u + threadIdx.x;
@@ -236,6 +237,7 @@ template <typename T, int K, int MODE, typename I>
 __global__ void __launch_bounds__(256)
 compress_nchw_vec(const T* __restrict__ x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int Hp,
                   int Wp, long long total) {
+    pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
     constexpr bool RELU = MODE != 0;
     constexpr int VW = VecTraits<T>::VW;
     const int WV = W / VW;
@@ -303,6 +305,7 @@ template <typename T, bool RELU>
 __global__ void __launch_bounds__(256)
 compress_generic(const T* x, T* __restrict__ z, T* y, int C, int H, int W, int k, int Hp, int Wp,
                  int nhwc, long long total) {
+    pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total) return;
     int c, p, q;

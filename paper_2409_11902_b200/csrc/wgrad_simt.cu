@@ -165,6 +165,7 @@ splitk_reduce4_kernel(const float4* __restrict__ partials, int splits, long long
     const int e = threadIdx.x % EL, sl = threadIdx.x / EL;
     const long long i = (long long)blockIdx.x * EL + e;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    pdl_wait();   // launched behind the kernel that writes the partial sums, possibly before it ends
     if (i < elems4) {
         int sp = sl;
         for (; sp + 3 * SL < splits; sp += 4 * SL) {       // four loads in flight
@@ -202,8 +203,8 @@ splitk_reduce4_kernel(const float4* __restrict__ partials, int splits, long long
 template <int SL>
 void launch_reduce4(const float* partials, int splits, long long e4, float* dw, cudaStream_t stream) {
     constexpr int EL = 256 / SL;
-    splitk_reduce4_kernel<SL><<<(unsigned)((e4 + EL - 1) / EL), 256, 0, stream>>>(
-        reinterpret_cast<const float4*>(partials), splits, e4, reinterpret_cast<float4*>(dw));
+    launch_after(splitk_reduce4_kernel<SL>, dim3((unsigned)((e4 + EL - 1) / EL)), dim3(256), 0, stream,
+                 reinterpret_cast<const float4*>(partials), splits, e4, reinterpret_cast<float4*>(dw));
 }
 
 }  // namespace

@@ -177,9 +177,6 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     unsigned char* smem_gen = tc2_smem + (smem_base - smem_u32(tc2_smem));
     const uint32_t a_base = smem_base, b_base = smem_base + kSlotsA * p.a_slot_bytes;
 
-    // The status block starts clean: CTA 0 resets it here, long before any wait of this launch
-    // can run out (a wait gives up only after 2^32 cycles).
-    if (blockIdx.x == 0 && tid == 0 && !p.keep_status) { p.status[0] = 0u; p.status[1] = 0u; }
 
     // ---------------------------------------------------------------- TMA producer
     // Warp 0 issues every copy. The stream of copies is: for each K-tile, the Z halo
@@ -274,6 +271,12 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         // (issuing the first round of them takes about 3 us; the first tile lands long before).
         __threadfence_block();
         bar_arrive(1, kThreads2);
+        // Everything up to here touched no global memory and may have run while the kernel before
+        // this one in the stream (the compress kernel that writes Z, say) was still finishing.
+        pdl_wait();
+        // The status block starts clean: CTA 0 resets it here, long before any wait of this launch
+        // can run out (a wait gives up only after 2^32 cycles).
+        if (blockIdx.x == 0 && lane == 0 && !p.keep_status) { p.status[0] = 0u; p.status[1] = 0u; }
         produce(true);
     }
     // Everything the MMAs may read but no copy ever writes must be finite (it only
@@ -433,6 +436,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         const bool add_to = kchunk > 0;      // later chunks add to what the earlier ones stored
+        if (kchunk == 0) pdl_wait();         // first global access of these warps (dW may still be read)
+        if (kchunk + 1 == nchunk_k && warp == 2 && lane == 0)
+            pdl_launch_dependents();         // the split-K reduction may be brought onto the SMs now
         {
             tc_fence_after();
             const int quarter = warp & 3;            // the TMEM lanes this warp may read
@@ -1037,7 +1043,7 @@ static ac_status launch_tc2_any(const Dims& d, bool collapse, const void* z, con
         if (st_ != AC_OK) return st_;
     }
     record_timing_hook(0, stream);
-    wgrad_tc2_kernel<<<p.groups * p.splits, kThreads2, g.smem_bytes, stream>>>(p);
+    launch_after(wgrad_tc2_kernel, dim3(p.groups * p.splits), dim3(kThreads2), g.smem_bytes, stream, p);
     record_timing_hook(1, stream);
     AC_CUDA_TRY(cudaGetLastError());
     if (p.collapse) {

@@ -168,6 +168,41 @@ def test_accumulate_adds_to_what_dw_holds(dtype, layout):
         assert e.value.status == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
 
 
+@pytest.mark.parametrize("layer", [(16, 128, 128, 28, 28), (8, 64, 64, 56, 56), (32, 512, 512, 8, 8)])
+def test_back_to_back_calls_see_each_others_results(layer):
+    """compress -> wgrad -> (reduce) queued without any synchronisation, inputs changing from call to
+    call: each kernel may be brought onto the GPU while the one before it is still finishing, and must
+    still read what that one wrote. Compared bit for bit with the same calls synchronised one by one."""
+    import torch
+    import paper_2409_11902_b200 as ac
+    N, Ci, Co, H, W = layer
+    d = D(N, Ci, Co, H, W, 3, 3, 1, 1, 2, "bf16", "nhwc")
+    g = torch.Generator(device="cuda").manual_seed(11)
+    xs = [torch.randn(d.x_shape, generator=g, device="cuda").relu().to(torch.bfloat16) for _ in range(4)]
+    dy = (torch.randn((N, d.Ho, d.Wo, Co), generator=g, device="cuda") * 1e-2).to(torch.bfloat16)
+    z = torch.empty(d.z_shape, dtype=torch.bfloat16, device="cuda")
+    dw = torch.empty(d.dw_shape, dtype=torch.float32, device="cuda")
+    ws = torch.empty(ac.ac_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+    refs = []
+    for x in xs:
+        ac.ac_compress(d, x, z)
+        torch.cuda.synchronize()
+        ac.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws)
+        torch.cuda.synchronize()
+        refs.append(dw.clone())
+    assert not torch.equal(refs[0], refs[1])
+    outs = []
+    for rnd in range(5):
+        for x in xs:
+            ac.ac_compress(d, x, z)
+            ac.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws)
+            outs.append(dw.clone())
+    torch.cuda.synchronize()
+    assert ac.ac_workspace_status(ws)[0] == 0
+    for i, o in enumerate(outs):
+        assert torch.equal(o, refs[i % 4]), i
+
+
 BOTTLENECK = [  # config 3: batch 128, bf16
     (128, 256, 64, 56, 56, 1, 1, 1, 0), (128, 64, 64, 56, 56, 3, 3, 1, 1),
     (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
