@@ -334,8 +334,14 @@ def run_ours(args):
     d2h = sum(p["dw"].numel() * 4 for p in pinned)
 
     def e2e_step():
-        for (name, d), p in zip(layers, pinned):
-            ac.ac_backward_step_host(d, p["x"], p["dy"], p["dw"], None, p["arena"])
+        # every layer's call on a stream of its own (the layers are independent and each has its own
+        # arena), so that one layer's device->host copy of dW runs while the next layer's inputs are
+        # still coming in: PCIe carries both directions at once
+        for s_, ((name, d), p) in zip(side, zip(layers, pinned)):
+            s_.wait_stream(stream)
+            ac.ac_backward_step_host(d, p["x"], p["dy"], p["dw"], None, p["arena"], stream=s_)
+        for s_ in side:
+            stream.wait_stream(s_)
     for _ in range(3):
         e2e_step()
     torch.cuda.synchronize()
