@@ -21,7 +21,10 @@ struct UnitPlan {
     bool ok;
 };
 
-inline UnitPlan plan_units(int Ci, int Co, int ntaps, int max_units) {
+// fill_rectangles: when the taps do not fit one CTA, let a CTA's tiles be any taps x channel-blocks
+// rectangle (not only taps of one channel block), chosen so that as few CTAs as possible are left
+// with fewer tiles than the others.
+inline UnitPlan plan_units(int Ci, int Co, int ntaps, int max_units, bool fill_rectangles = false) {
     UnitPlan u{};
     u.ok = false;
     if (Ci % 64 != 0 || Co % 64 != 0) return u;
@@ -40,6 +43,21 @@ inline UnitPlan plan_units(int Ci, int Co, int ntaps, int max_units) {
         u.taps_per_group = (ntaps + u.ntapgroups - 1) / u.ntapgroups;
         u.ntapgroups = (ntaps + u.taps_per_group - 1) / u.taps_per_group;
         u.cibs_per_group = 1;
+        if (fill_rectangles) {
+            // 9 taps in CTAs of 2 tiles: (2,2,2,2,1) taps of one block leaves every fifth CTA half
+            // empty; 1 tap x 2 blocks fills them all. Ties go to more taps (a smaller input tile).
+            long long best_slots = (long long)u.ntapgroups * u.taps_per_group * u.ncib_total;
+            for (int t = U; t >= 1; --t) {
+                int c = U / t < u.ncib_total ? U / t : u.ncib_total;
+                if (c < 1 || t * c > max_units) continue;
+                const int tg = (ntaps + t - 1) / t, cg = (u.ncib_total + c - 1) / c;
+                const long long slots = (long long)tg * t * cg * c;      // tile slots over all CTAs
+                if (slots < best_slots) {
+                    best_slots = slots;
+                    u.taps_per_group = t; u.ntapgroups = tg; u.cibs_per_group = c;
+                }
+            }
+        }
     }
     u.units = u.cibs_per_group * u.taps_per_group;
     if (u.units > max_units) return u;

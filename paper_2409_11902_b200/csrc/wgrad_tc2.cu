@@ -591,6 +591,7 @@ __global__ void bounded_wait_selftest_kernel(uint32_t* status, long long limit_c
 // ------------------------------------------------------------------ host side
 struct Tc2Geom {
     Tc2Params p;
+    double cta_cycles;   // the cost model's main-loop time of the busiest CTA
     uint32_t smem_bytes;
     int uspan, vspan;
     double k_eff;
@@ -707,14 +708,14 @@ int min_flat_pitch(int J, int lo, int hi, int ext) {
     return J + (hi - lo);
 }
 
-Tc2Geom build_geom2(const Dims& d, bool collapse) {
+Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles) {
     Tc2Geom g{};
     Tc2Params& p = g.p;
     g.ok = false;
     if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
     if (d.k % d.sh != 0 || d.k % d.sw != 0) return g;      // class rows advance Z by exactly one row
     if (d.R * d.S > 64 || d.R > 16 || d.S > 16) return g;
-    const UnitPlan up = plan_units(d.Ci, d.Co, d.R * d.S, kMaxUnits2);
+    const UnitPlan up = plan_units(d.Ci, d.Co, d.R * d.S, kMaxUnits2, fill_rectangles);
     if (!up.ok) return g;
     p.c_h = d.k / d.sh; p.c_w = d.k / d.sw;
     p.ncls = p.c_h * p.c_w;
@@ -893,8 +894,22 @@ Tc2Geom build_geom2(const Dims& d, bool collapse) {
     }
     g.smem_bytes = kSlotsA * p.a_slot_bytes + p.slotsB * p.b_slot_bytes + 1024;
     if (g.smem_bytes < 120 * 1024) g.smem_bytes = 120 * 1024;   // one CTA per SM: TMEM is not shared
+    g.cta_cycles = best_cost;
     g.ok = true;
     return g;
+}
+
+// Two ways to deal the accumulator tiles to CTAs (see plan_units): taps of one channel block per
+// CTA, or taps x channel-blocks rectangles that leave no CTA half empty but need a larger input
+// tile in shared memory (hence shorter K-tiles when several copies of it are kept). The cost
+// model's time for the busiest CTA decides.
+Tc2Geom build_geom2(const Dims& d, bool collapse) {
+    const Tc2Geom a = build_geom2_with(d, collapse, false);
+    if (collapse) return a;
+    const Tc2Geom b = build_geom2_with(d, collapse, true);
+    if (!a.ok) return b;
+    if (!b.ok) return a;
+    return b.cta_cycles < a.cta_cycles ? b : a;
 }
 
 // The geometry is pure arithmetic on the descriptor but not free (the pairing search):
