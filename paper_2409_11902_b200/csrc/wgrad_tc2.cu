@@ -884,6 +884,13 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles) {
     int splits = kNumSMs / p.groups;
     if (splits < 1) splits = 1;
     if (splits > p.ktiles) splits = p.ktiles;
+    {
+        // K-tiles are dealt out whole, so the busiest slice has ceil(ktiles / splits) of them: no more
+        // slices than that number needs (896 tiles: 128 slices of 7 finish when 148 slices of 6 or 7
+        // do, with fewer partial sums to write and reduce, and leave SMs to other streams)
+        const int per_slice = (p.ktiles + splits - 1) / splits;
+        splits = (p.ktiles + per_slice - 1) / per_slice;
+    }
     p.splits = splits;
     p.chunk_kt = 0;
     if (d.max_chain > 0) {
