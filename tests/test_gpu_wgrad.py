@@ -50,6 +50,40 @@ def test_wgrad_matches_checker(case, dtype, layout):
     assert err <= TOL_DW[dtype], err
 
 
+def _random_cases(n, seed, tensor_shapes=False):
+    """tensor_shapes: channel counts and stride/k pairs that the tensor-core kernels take."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < n:
+        chans = [64, 128, 192, 256] if tensor_shapes else [8, 24, 64, 64, 128, 192]
+        Ci, Co = (int(rng.choice(chans)) for _ in range(2))
+        H, W = int(rng.integers(1, 21)), int(rng.integers(1, 21))
+        R, S = int(rng.choice([1, 3, 5])), int(rng.choice([1, 3, 5]))
+        stride, pad, k = int(rng.integers(1, 4)), int(rng.integers(0, 3)), int(rng.choice([1, 2, 2, 3, 4]))
+        if tensor_shapes:
+            k = int(rng.choice([1, 2, 2, 4, 8]))
+            stride = int(rng.choice([s for s in (1, 2, 4) if k % s == 0] + [2]))
+        if H + 2 * pad < R or W + 2 * pad < S:
+            continue
+        cases.append((int(rng.integers(1, 6)), Ci, Co, H, W, R, S, stride, pad, k,
+                      str(rng.choice(["bf16", "f32"])), str(rng.choice(["nhwc", "nchw"]))))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_cases(48, seed=2024) + _random_cases(64, seed=7, tensor_shapes=True))
+def test_random_descriptors_match_checker(case):
+    """Seeded random layer shapes over every dtype/layout pair: whichever kernel the planner picks
+    (TMA-fed, producer-fed, staged, fp32 FMA) must meet the bound; rectangular filters, strides that
+    do not divide k, maps smaller than the filter's reach and single-pixel maps included."""
+    d = D(*case)
+    err, got, want = wgrad_error_full(d)
+    assert np.isfinite(got).all()
+    if np.linalg.norm(want) == 0.0:
+        assert not got.any()
+    else:
+        assert err <= TOL_DW[case[10]], (case, err)
+
+
 def test_k1_equals_uncompressed_dw():
     """k = 1: Z is X, so the result must be the ordinary weight gradient."""
     import oracle
