@@ -152,6 +152,12 @@ ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z
  *                   must not share a workspace.
  * Returns AC_ERR_WORKSPACE_TOO_SMALL / AC_ERR_MISALIGNED / AC_ERR_INVALID_ARG
  * before launching anything. Results are deterministic (fixed summation order).
+ * Stream semantics are the ordinary ones. Internally the main kernel and the
+ * split-K reduction are launched with CUDA's programmatic stream
+ * serialization: if the kernel before them in the stream allows it (the
+ * library's own compress kernels do), they are brought onto the GPU while
+ * that kernel is finishing, but touch global memory only once it has
+ * completed and its writes are visible.
  */
 ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc *desc, const void *z,
                                      const void *dy, float *dw, void *workspace,
