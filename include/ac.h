@@ -42,7 +42,7 @@ extern "C" {
 typedef enum {
     AC_OK = 0,
     AC_ERR_INVALID_ARG = 1,         /* NULL pointer, non-positive size, bad enum, empty output */
-    AC_ERR_UNSUPPORTED = 2,         /* valid problem this build cannot run */
+    AC_ERR_UNSUPPORTED = 2,         /* valid problem the library cannot run */
     AC_ERR_MISALIGNED = 3,          /* a tensor or workspace pointer is not 16-byte aligned */
     AC_ERR_WORKSPACE_TOO_SMALL = 4, /* workspace_bytes < ac_workspace_bytes_min(desc) */
     AC_ERR_CUDA = 5,                /* a CUDA runtime call failed (launch, copy, attribute) */

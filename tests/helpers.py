@@ -9,7 +9,7 @@ from paper_2409_11902_b200 import synth
 
 CANARY = 0x5A
 
-# Tolerances (stated by the benchmark spec for this path):
+# Tolerances of this path:
 #   fp32 compress: max relative error <= 1e-6 (relative to the block's mean |x|)
 #   bf16 compress: one rounding to bf16 (half an ulp = 2^-9 .. 2^-8 relative) on top
 #   dW: relative Frobenius error <= 1e-5 (fp32 inputs), <= 1e-2 (bf16 inputs, fp32 accumulate)
