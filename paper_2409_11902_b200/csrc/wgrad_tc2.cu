@@ -692,17 +692,20 @@ bool plan_pairs(const Dims& d, int c_h, int c_w, int umin, int vmin, int uspan, 
 // cells of the next one, which is harmless exactly when both the coordinate it wants and the one it
 // gets are outside [0, ext): the tensor map fills those with the convolution's zero padding either
 // way. For a padded 3x3 layer this lets the right halo of one line double as the left halo of the
-// next (P = J + 1 instead of J + 2).
-int min_flat_pitch(int J, int lo, int hi, int ext) {
+// next (P = J + 1 instead of J + 2). With a partial last block the tile is also kept in a copy
+// that ends one coordinate earlier (ext - 1, see Tc2Params::nvar); `also_shorter` asks for a pitch
+// that is right for both.
+int min_flat_pitch(int J, int lo, int hi, int ext, bool also_shorter) {
     for (int P = J; P < J + (hi - lo); ++P) {
         bool ok = true;
-        for (int c = 0; c < J && ok; ++c)
-            for (int v = lo; v <= hi && ok; ++v) {
-                const int t = c + v - lo;
-                if (t < P) continue;
-                const int want = c + v, got = lo + t - P;
-                ok = (want < 0 || want >= ext) && (got < 0 || got >= ext) && t - P < P;
-            }
+        for (int e = ext; e >= ext - (also_shorter ? 1 : 0) && ok; --e)
+            for (int c = 0; c < J && ok; ++c)
+                for (int v = lo; v <= hi && ok; ++v) {
+                    const int t = c + v - lo;
+                    if (t < P) continue;
+                    const int want = c + v, got = lo + t - P;
+                    ok = (want < 0 || want >= e) && (got < 0 || got >= e) && t - P < P;
+                }
         if (ok) return P;
     }
     return J + (hi - lo);
@@ -809,9 +812,9 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles) {
         while (p.tmem_cols < (uint32_t)(p.cu_cap * up.BN)) p.tmem_cols *= 2;
         p.slice_elems = (long long)up.ncob * up.ncib_total * total * up.BN * up.CB;
     }
-    if (!p.pair_mode && p.nvar == 1) {
-        p.Wzq = min_flat_pitch(Jc, vmin, vmax, d.Wp);
-        rows_whole = min_flat_pitch(I, umin, umax, d.Hp);
+    if (!p.pair_mode) {
+        p.Wzq = min_flat_pitch(Jc, vmin, vmax, d.Wp, var_used[1] || var_used[3]);
+        rows_whole = min_flat_pitch(I, umin, umax, d.Hp, var_used[2] || var_used[3]);
     }
     int best_Ic = 0, best_sb = 0, best_NB = 1;
     double best_cost = 1e30, best_eff = 0.0;
