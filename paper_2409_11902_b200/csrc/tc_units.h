@@ -24,7 +24,10 @@ struct UnitPlan {
 // fill_rectangles: when the taps do not fit one CTA, let a CTA's tiles be any taps x channel-blocks
 // rectangle (not only taps of one channel block), chosen so that as few CTAs as possible are left
 // with fewer tiles than the others.
-inline UnitPlan plan_units(int Ci, int Co, int ntaps, int max_units, bool fill_rectangles = false) {
+// bn_cap: widest output-channel block considered (a narrower one leaves more shared memory to the
+// input tile).
+inline UnitPlan plan_units(int Ci, int Co, int ntaps, int max_units, bool fill_rectangles = false,
+                           int bn_cap = 256) {
     UnitPlan u{};
     u.ok = false;
     if (Ci % 64 != 0 || Co % 64 != 0) return u;
@@ -32,6 +35,7 @@ inline UnitPlan plan_units(int Ci, int Co, int ntaps, int max_units, bool fill_r
     u.ncgpc = u.CB / 8;
     u.ncib_total = Ci / u.CB;
     u.BN = Co <= 256 ? Co : (Co % 256 == 0 ? 256 : (Co % 128 == 0 ? 128 : 64));
+    while (u.BN > bn_cap && u.BN % 128 == 0) u.BN /= 2;
     u.ncob = Co / u.BN;
     const int U = 512 / u.BN;
     if (ntaps <= U) {

@@ -711,14 +711,14 @@ int min_flat_pitch(int J, int lo, int hi, int ext, bool also_shorter) {
     return J + (hi - lo);
 }
 
-Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles) {
+Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int bn_cap = 256) {
     Tc2Geom g{};
     Tc2Params& p = g.p;
     g.ok = false;
     if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
     if (d.k % d.sh != 0 || d.k % d.sw != 0) return g;      // class rows advance Z by exactly one row
     if (d.R * d.S > 64 || d.R > 16 || d.S > 16) return g;
-    const UnitPlan up = plan_units(d.Ci, d.Co, d.R * d.S, kMaxUnits2, fill_rectangles);
+    const UnitPlan up = plan_units(d.Ci, d.Co, d.R * d.S, kMaxUnits2, fill_rectangles, bn_cap);
     if (!up.ok) return g;
     p.c_h = d.k / d.sh; p.c_w = d.k / d.sw;
     p.ncls = p.c_h * p.c_w;
@@ -917,9 +917,16 @@ Tc2Geom build_geom2(const Dims& d, bool collapse) {
     const Tc2Geom a = build_geom2_with(d, collapse, false);
     if (collapse) return a;
     const Tc2Geom b = build_geom2_with(d, collapse, true);
-    if (!a.ok) return b;
-    if (!b.ok) return a;
-    return b.cta_cycles < a.cta_cycles ? b : a;
+    Tc2Geom best = !a.ok ? b : (!b.ok ? a : (b.cta_cycles < a.cta_cycles ? b : a));
+    if (best.ok && best.p.nvar > 1 && best.p.BN > 128) {
+        // several copies of the input tile (partial pooling blocks): a narrower output-channel block
+        // may leave room for longer K-tiles
+        for (int fill = 0; fill < 2; ++fill) {
+            const Tc2Geom c = build_geom2_with(d, collapse, fill != 0, 128);
+            if (c.ok && c.cta_cycles < best.cta_cycles) best = c;
+        }
+    }
+    return best;
 }
 
 // The geometry is pure arithmetic on the descriptor but not free (the pairing search):
