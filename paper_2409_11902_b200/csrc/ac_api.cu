@@ -94,6 +94,11 @@ WgradPlan plan_wgrad(const Dims& d) {
         plan_staged(d, &p);
         return p;
     }
+    if (gather_supported(d)) {
+        WgradPlan p{};
+        plan_gather(d, &p);
+        return p;
+    }
     if (tc_supported(d)) {
         WgradPlan p{};
         p.path = PATH_TC;
@@ -119,7 +124,7 @@ size_t ac_workspace_bytes_min(const ac_conv_desc* desc) {
     Dims d;
     if (make_dims(desc, true, &d) != AC_OK) return 0;
     const WgradPlan p = plan_wgrad(d);
-    return p.path == PATH_STAGED ? plan_wgrad_unstaged(d).bytes : p.bytes;
+    return p.path == PATH_STAGED || p.path == PATH_GATHER ? plan_wgrad_unstaged(d).bytes : p.bytes;
 }
 
 ac_status ac_compress(const ac_conv_desc* desc, const void* x, void* z, void* y_out, void* stream) {
@@ -151,11 +156,12 @@ ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, co
     if (!aligned16(z) || !aligned16(dy) || !aligned16(dw) || !aligned16(workspace))
         return AC_ERR_MISALIGNED;
     WgradPlan p = plan_wgrad(d);
-    if (p.path == PATH_STAGED && workspace_bytes < p.bytes) p = plan_wgrad_unstaged(d);
+    if ((p.path == PATH_STAGED || p.path == PATH_GATHER) && workspace_bytes < p.bytes) p = plan_wgrad_unstaged(d);
     if (workspace_bytes < p.bytes) return AC_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (p.path == PATH_TC2) return launch_wgrad_tc2(d, p, z, dy, dw, workspace, s);   // resets the status itself
     if (p.path == PATH_STAGED) return launch_wgrad_staged(d, p, z, dy, dw, workspace, s);
+    if (p.path == PATH_GATHER) return launch_wgrad_gather(d, p, z, dy, dw, workspace, s);
     AC_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBlockBytes, s));
     if (p.path == PATH_TC) return launch_wgrad_tc(d, p, z, dy, dw, workspace, s);
     return launch_wgrad_simt(d, p, z, dy, dw, workspace, s);
@@ -256,6 +262,10 @@ ac_status ac_wgrad_plan_info(const ac_conv_desc* desc, ac_plan_info* info) {
     }
     if (staged_supported(d)) {
         staged_plan_info(d, info);
+        return AC_OK;
+    }
+    if (gather_supported(d)) {
+        gather_plan_info(d, info);
         return AC_OK;
     }
     if (tc_supported(d)) {

@@ -38,7 +38,7 @@ ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* out);
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---- wgrad planning (pure host arithmetic; decides kernel and split-K) ------
-enum WgradPath { PATH_SIMT = 0, PATH_TC = 1, PATH_TC2 = 2, PATH_STAGED = 3 };
+enum WgradPath { PATH_SIMT = 0, PATH_TC = 1, PATH_TC2 = 2, PATH_STAGED = 3, PATH_GATHER = 4 };
 
 struct WgradPlan {
     int path;        // WgradPath
@@ -81,6 +81,12 @@ void plan_staged(const Dims& d, WgradPlan* p);
 void staged_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                              float* dw, void* workspace, cudaStream_t stream);
+// few input channels: the operand gathered into a [positions][taps x channels] matrix (wgrad_staged.cu)
+bool gather_supported(const Dims& d);
+void plan_gather(const Dims& d, WgradPlan* p);
+void gather_plan_info(const Dims& d, ac_plan_info* info);
+ac_status launch_wgrad_gather(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
+                              float* dw, void* workspace, cudaStream_t stream);
 size_t tc2_collapsed_workspace_bytes(const Dims& d, int* tiles_collapsed, int* tiles_dense);
 ac_status launch_wgrad_tc2_collapsed(const Dims& d, const void* z, const void* dy, float* dw,
                                      void* workspace, cudaStream_t stream);

@@ -23,7 +23,20 @@
 //  * NCHW inputs (either dtype). The kernel's tap shift needs channels innermost, so the staging
 //    pass also transposes each image from [C][H*W] to [H*W][C]; the kernel then produces dW as
 //    [C_out][R][S][C_in] in the workspace and a last small pass permutes it to [C_out][C_in][R][S].
+//
+//  * Few input channels (the 3-channel stem convolution; bf16 NHWC). The kernel's unit is a 64-channel
+//    vector per cell, which three channels cannot fill. Here the staging pass gathers, for every output
+//    position, the inflated and zero-padded values all its taps read into one row of a matrix
+//    G[position][(tap, channel)], padded to a multiple of 64 columns; the weight gradient is then the
+//    1x1 problem dW'[co][column] = sum over positions of dY[position][co] * G[position][column] on the
+//    output map, which the kernel takes as it is, and a last small pass copies the columns to dW.
+//    When both strides are multiples of k and k divides H and W, output (ho, wo) reads the pooled
+//    element Z[ho*s_h/k + u][wo*s_w/k + v] with u = floor((r - p_h)/k), v = floor((s - p_w)/k) for
+//    EVERY position, so taps with equal (u, v) have equal columns: G then keeps one column per distinct
+//    (u, v, channel) (7x7, stride 2, pad 3, k = 2: 16 shifts instead of 49 taps; 48 columns instead of
+//    147, a third of the bytes written and read) and the last pass copies each column to all its taps.
 #include "ac_common.h"
+#include "tc_units.h"
 
 namespace ac {
 namespace {
@@ -185,6 +198,129 @@ permute_dw_kernel(const float* __restrict__ src, float* __restrict__ dst, int Ci
     dst[i] = src[(co * RS + t) * Ci + ci];
 }
 
+// ---- few input channels: gathered operand ------------------------------------------------------
+struct GatherParams {
+    int Ci, H, W, Hp, Wp, Ho, Wo, k;
+    int sh, sw, ph, pw;
+    int collapsed;      // 1: one column per distinct Z shift (u, v); 0: one per tap (r, s)
+    int mh, mw;         // collapsed: Z rows / columns per output row / column (s_h / k, s_w / k)
+    int u0, v0;         // collapsed: first shift
+    int nb;             // shifts (collapsed) or taps per row of shifts / taps: nV or S
+    int cols, Mp;       // valid columns (shifts or taps, times C_in), row length of G (multiple of 64)
+    long long groups;   // positions * Mp / 8
+};
+
+// G[position][column], eight columns (one 16-byte vector) per thread. Z is read element by element
+// (it is k^2 times smaller than what is written and stays in L2); consecutive threads write
+// consecutive vectors.
+__global__ void __launch_bounds__(256)
+gather_kernel(const unsigned short* __restrict__ z, uint4* __restrict__ g, const GatherParams p) {
+    __shared__ int tab[256];    // column -> a | b << 8 | channel << 16, or -1 behind the last column
+    for (int j = threadIdx.x; j < p.Mp; j += 256) {
+        int e = -1;
+        if (j < p.cols) {
+            const int t = j / p.Ci, ci = j - t * p.Ci, a = t / p.nb, b = t - a * p.nb;
+            e = a | (b << 8) | (ci << 16);
+        }
+        tab[j] = e;
+    }
+    __syncthreads();
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= p.groups) return;
+    const int G = p.Mp / 8;
+    const long long pos = idx / G;
+    const int j0 = (int)(idx - pos * G) * 8;
+    const int wo = (int)(pos % p.Wo);
+    const long long t1 = pos / p.Wo;
+    const int ho = (int)(t1 % p.Ho);
+    const long long n = t1 / p.Ho;
+    const unsigned short* zn = z + n * p.Hp * p.Wp * p.Ci;
+    const int rb = p.collapsed ? ho * p.mh + p.u0 : ho * p.sh - p.ph;
+    const int cb = p.collapsed ? wo * p.mw + p.v0 : wo * p.sw - p.pw;
+    unsigned short v[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int e = tab[j0 + q];
+        unsigned short val = 0;
+        if (e >= 0) {
+            int zr = rb + (e & 255), zc = cb + ((e >> 8) & 255);
+            bool in;
+            if (p.collapsed) {
+                in = zr >= 0 && zr < p.Hp && zc >= 0 && zc < p.Wp;
+            } else {
+                in = zr >= 0 && zr < p.H && zc >= 0 && zc < p.W;      // coordinates of the inflated map
+                zr /= p.k;
+                zc /= p.k;
+            }
+            if (in) val = __ldg(zn + ((long long)zr * p.Wp + zc) * p.Ci + (e >> 16));
+        }
+        v[q] = val;
+    }
+    g[idx] = make_uint4(v[0] | (uint32_t)v[1] << 16, v[2] | (uint32_t)v[3] << 16, v[4] | (uint32_t)v[5] << 16,
+                        v[6] | (uint32_t)v[7] << 16);
+}
+
+// dW[co][r][s][ci] = dW'[co][column of (r, s, ci)]
+__global__ void __launch_bounds__(256)
+scatter_columns_kernel(const float* __restrict__ src, float* __restrict__ dw, const GatherParams p, int R, int S,
+                       long long total) {
+    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (i >= total) return;
+    const int row = R * S * p.Ci;
+    const long long co = i / row;
+    int col = (int)(i - co * row);
+    if (p.collapsed) {
+        const int t = col / p.Ci, ci = col - t * p.Ci, r = t / S, s = t - r * S;
+        const int iu = floor_div_i(r - p.ph, p.k) - p.u0, iv = floor_div_i(s - p.pw, p.k) - p.v0;
+        col = (iu * p.nb + iv) * p.Ci + ci;
+    }
+    dw[i] = src[co * p.Mp + col];
+}
+
+struct GatherGeom {
+    bool ok;
+    GatherParams p;
+    Dims in;       // the 1x1 problem on the output map
+};
+
+GatherGeom gather_geom(const Dims& d) {
+    GatherGeom g{};
+    if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
+    if (d.Ci >= 64 || d.Co % 64 != 0) return g;
+    if (d.R > 255 || d.S > 255) return g;
+    GatherParams& p = g.p;
+    p.Ci = d.Ci; p.H = d.H; p.W = d.W; p.Hp = d.Hp; p.Wp = d.Wp; p.Ho = d.Ho; p.Wo = d.Wo; p.k = d.k;
+    p.sh = d.sh; p.sw = d.sw; p.ph = d.ph; p.pw = d.pw;
+    p.collapsed = d.k > 1 && d.sh % d.k == 0 && d.sw % d.k == 0 && d.H % d.k == 0 && d.W % d.k == 0;
+    int na = d.R;
+    p.nb = d.S;
+    if (p.collapsed) {
+        p.mh = d.sh / d.k; p.mw = d.sw / d.k;
+        p.u0 = floor_div_i(-d.ph, d.k); p.v0 = floor_div_i(-d.pw, d.k);
+        na = floor_div_i(d.R - 1 - d.ph, d.k) - p.u0 + 1;
+        p.nb = floor_div_i(d.S - 1 - d.pw, d.k) - p.v0 + 1;
+    }
+    const long long cols = (long long)na * p.nb * d.Ci;
+    if (cols > 256) return g;
+    p.cols = (int)cols;
+    p.Mp = (p.cols + 63) / 64 * 64;
+    const long long positions = d.K();
+    if (positions * p.Mp >= (1ll << 40)) return g;
+    p.groups = positions * (p.Mp / 8);
+    if ((p.groups + 255) / 256 >= (1ll << 31)) return g;
+    Dims in = d;
+    in.Ci = p.Mp;
+    in.H = in.Hp = d.Ho;
+    in.W = in.Wp = d.Wo;
+    in.R = in.S = 1;
+    in.sh = in.sw = 1;
+    in.ph = in.pw = 0;
+    in.k = 1;
+    g.in = in;
+    g.ok = tc2_supported(in, nullptr);
+    return g;
+}
+
 inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 // fp32 results: at most this many MMA instructions add into an accumulator before the kernel
@@ -342,6 +478,43 @@ ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z,
     if (d.layout == AC_NHWC) return AC_OK;
     const long long total = d.dw_elems();
     permute_dw_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(out_nhwc, dw, d.Ci, d.R * d.S, total);
+    AC_CUDA_TRY(cudaGetLastError());
+    return AC_OK;
+}
+
+bool gather_supported(const Dims& d) { return gather_geom(d).ok; }
+
+void plan_gather(const Dims& d, WgradPlan* pl) {
+    const GatherGeom g = gather_geom(d);
+    plan_tc2(g.in, pl);
+    pl->path = PATH_GATHER;
+    pl->st_off_z = up256(pl->bytes);
+    pl->st_off_dy = pl->st_off_z;
+    pl->st_off_dw = pl->st_off_z + up256((size_t)g.in.z_elems() * 2);
+    pl->st_off_small = pl->st_off_dw;
+    pl->bytes = pl->st_off_dw + up256((size_t)g.in.dw_elems() * 4);
+}
+
+void gather_plan_info(const Dims& d, ac_plan_info* info) {
+    const GatherGeom g = gather_geom(d);
+    tc2_plan_info(g.in, info);
+    info->tensor_core = 5;
+}
+
+ac_status launch_wgrad_gather(const Dims& d, const WgradPlan& pl, const void* z, const void* dy, float* dw,
+                              void* workspace, cudaStream_t stream) {
+    const GatherGeom g = gather_geom(d);
+    if (!g.ok) return AC_ERR_UNSUPPORTED;
+    char* ws = static_cast<char*>(workspace);
+    uint4* gm = reinterpret_cast<uint4*>(ws + pl.st_off_z);
+    float* dw_cols = reinterpret_cast<float*>(ws + pl.st_off_dw);
+    gather_kernel<<<(unsigned)((g.p.groups + 255) / 256), 256, 0, stream>>>(
+        static_cast<const unsigned short*>(z), gm, g.p);
+    AC_CUDA_TRY(cudaGetLastError());
+    const ac_status st = launch_wgrad_tc2(g.in, pl, gm, dy, dw_cols, workspace, stream);
+    if (st != AC_OK) return st;
+    const long long total = d.dw_elems();
+    scatter_columns_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(dw_cols, dw, g.p, d.R, d.S, total);
     AC_CUDA_TRY(cudaGetLastError());
     return AC_OK;
 }

@@ -153,7 +153,7 @@ def test_plan_info_respects_hardware_limits(ac):
     # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
     for d in (ac.ConvDesc(8, 24, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw"),
               ac.ConvDesc(8, 64, 40, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
-              ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc"),
+              ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "f32", "nhwc"),
               ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (3, 3), (1, 1), 2, "bf16", "nhwc")):
         assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 0
     # fp32 NHWC goes to the tensor cores as six bf16 products: the same kernel on six times the
@@ -178,82 +178,34 @@ def test_plan_info_respects_hardware_limits(ac):
         assert ac.ac_workspace_bytes(dn) == (256 + info["splits"] * dw_bytes + (z6 + g6) * mult // 6 + dw_bytes)
 
 
-def test_binding_fails_loudly_without_the_library(ac, monkeypatch):
-    monkeypatch.setattr(ac.api, "_lib", None)
-    monkeypatch.setattr(ac.api, "_LIB_PATH", "/nonexistent/libac.so")
-    with pytest.raises(ImportError):
-        ac.ac_workspace_bytes(ac.ConvDesc(1, 8, 8, 8, 8))
-
-
-def test_plan_info_respects_hardware_limits(ac):
-    """Host-side planning of the tensor-core path: shared memory, tensor memory
-    and pipeline depth stay inside what one SM has, for every benchmark layer."""
-    shapes = [
-        (64, 64, 64, 56, 56, 3, 3, 1, 1), (64, 128, 128, 28, 28, 3, 3, 1, 1),
-        (64, 256, 256, 14, 14, 3, 3, 1, 1), (64, 512, 512, 7, 7, 3, 3, 1, 1),
-        (64, 512, 512, 8, 8, 3, 3, 1, 1), (128, 256, 64, 56, 56, 1, 1, 1, 0),
-        (128, 64, 256, 56, 56, 1, 1, 1, 0), (128, 128, 128, 56, 56, 3, 3, 2, 1),
-        (256, 128, 128, 64, 64, 3, 3, 1, 1), (256, 1024, 2048, 14, 14, 1, 1, 2, 0),
-        (8, 64, 64, 30, 30, 7, 7, 2, 3), (2, 192, 320, 9, 40, 3, 3, 1, 1),
-    ]
-    for N, ci, co, H, W, R, S, st, pd in shapes:
-        for k in (1, 2, 4, 8):
-            d = ac.ConvDesc(N, ci, co, H, W, R, S, (st, st), (pd, pd), k, "bf16", "nhwc")
-            i = ac.ac_wgrad_plan_info(d)
-            assert i["tensor_core"] in (1, 2), d
-            assert 2 <= i["stages"] <= 8
-            assert i["smem_bytes"] <= 227 * 1024
-            assert i["tmem_columns"] in (32, 64, 128, 256, 512)
-            assert i["units_per_cta"] * i["block_n"] <= i["tmem_columns"]
-            assert i["k_tile"] % 16 == 0
-            if i["tensor_core"] == 1:
-                assert i["k_tile"] >= i["band_rows"] * i["row_pitch"]
-                assert i["row_pitch"] >= d.Wo
-            else:   # per class: (band_rows / c_h) class rows of row_pitch >= Wo / c_w positions
-                c_h, c_w = k // st, k // st
-                assert i["phases"] == c_h * c_w <= 64
-                assert i["k_tile"] >= (i["band_rows"] // c_h) * i["row_pitch"]
-                assert i["row_pitch"] >= -(-d.Wo // c_w)
-            assert 1 <= i["splits"] <= d.N * -(-d.Ho // i["band_rows"])
-            assert i["ctas"] == i["splits"] * i["groups"]
-            want = 256 + (i["splits"] * 4 * co * ci * R * S if i["splits"] > 1 else 0)
-            assert ac.ac_workspace_bytes(d) == want
-    # 64 input channels, 3x3, k = 2: the nine taps pair up into five accumulator tiles in one CTA
-    i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 64, 64, 56, 56, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
-    assert (i["tensor_core"], i["units_per_cta"], i["groups"]) == (2, 5, 1)
-    # k = 8 at stride 1: 64 output classes, still the TMA-fed kernel
-    i = ac.ac_wgrad_plan_info(ac.ConvDesc(256, 128, 128, 64, 64, 3, 3, (1, 1), (1, 1), 8, "bf16", "nhwc"))
-    assert (i["tensor_core"], i["phases"]) == (2, 64)
-    # a map that k does not divide (partial pooling blocks) is still taken by the TMA-fed kernel
-    i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 512, 512, 7, 7, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
-    assert i["tensor_core"] == 2
-    # a stride that does not divide k goes to the producer-fed tensor-core kernel
-    i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 28, 28, 3, 3, (2, 2), (1, 1), 1, "bf16", "nhwc"))
-    assert i["tensor_core"] == 1
-    # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
-    for d in (ac.ConvDesc(8, 24, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw"),
-              ac.ConvDesc(8, 64, 40, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
-              ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc"),
-              ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (3, 3), (1, 1), 2, "bf16", "nhwc")):
-        assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 0
-    # fp32 NHWC goes to the tensor cores as six bf16 products: the same kernel on six times the
-    # images, with room for the split operands in the workspace
-    d32 = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nhwc")
-    d16 = ac.ConvDesc(48, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
-    i32, i16 = ac.ac_wgrad_plan_info(d32), ac.ac_wgrad_plan_info(d16)
-    assert i32["tensor_core"] == 3 and i16["tensor_core"] == 2
-    # ... except that the K-slices are shorter (bounded accumulation chains), hence more of them
-    varies = ("tensor_core", "splits", "ctas")
-    assert {k: v for k, v in i32.items() if k not in varies} == {k: v for k, v in i16.items() if k not in varies}
-    assert i32["splits"] >= i16["splits"] and i32["ctas"] == i32["splits"] * i32["groups"]
-    z6 = 48 * 64 * 16 * 16 * 2
-    g6 = 48 * 64 * 32 * 32 * 2
-    dw_bytes = 64 * 64 * 9 * 4
-    assert ac.ac_workspace_bytes(d32) == 256 + i32["splits"] * dw_bytes + z6 + g6
-    # NCHW inputs are transposed on the way: same kernel, plus room for its NHWC-ordered dW
-    for dt, mult in (("bf16", 1), ("f32", 6)):
-        dn = ac.ConvDesc(8, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, dt, "nchw")
-        di = ac.ConvDesc(8 * mult, 64, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
-        assert ac.ac_wgrad_plan_info(dn)["tensor_core"] == 3
-        assert ac.ac_workspace_bytes(dn) == (ac.ac_workspace_bytes(di) + (z6 + g6) * mult // 6
-                                             + 64 * 64 * 9 * 4)
+def test_few_input_channels_are_gathered_for_the_tensor_cores(ac):
+    """bf16 NHWC layers with fewer than 64 input channels (the 3-channel stem): the operand is
+    gathered into a [positions][taps x channels] matrix in the workspace and the tensor-core kernel
+    runs the equivalent 1x1 problem on the output map."""
+    def inner(N, cols, co, Ho, Wo):
+        return ac.ConvDesc(N, cols, co, Ho, Wo, 1, 1, (1, 1), (0, 0), 1, "bf16", "nhwc")
+    # 7x7, stride 2, pad 3, k = 2, k | H: taps collapse to 4 x 4 shifts -> 48 columns, padded to 64
+    d = ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc")
+    i = ac.ac_wgrad_plan_info(d)
+    assert i["tensor_core"] == 5
+    di = inner(8, 64, 64, 16, 16)
+    ii = ac.ac_wgrad_plan_info(di)
+    assert ii["tensor_core"] == 2 and {k: v for k, v in i.items() if k != "tensor_core"} == \
+        {k: v for k, v in ii.items() if k != "tensor_core"}
+    assert ac.ac_workspace_bytes(d) == ac.ac_workspace_bytes(di) + 8 * 16 * 16 * 64 * 2 + 64 * 64 * 4
+    # an odd map cannot collapse (the partial last block): one column per tap, 147 -> 192
+    d = ac.ConvDesc(8, 3, 64, 31, 31, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc")
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 5
+    assert ac.ac_workspace_bytes(d) == ac.ac_workspace_bytes(inner(8, 192, 64, 16, 16)) + 8 * 16 * 16 * 192 * 2 + 64 * 192 * 4
+    # stride 1 at k = 2: no collapse either; 3x3x3 = 27 columns -> 64
+    d = ac.ConvDesc(4, 3, 128, 20, 20, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 5
+    assert ac.ac_workspace_bytes(d) == ac.ac_workspace_bytes(inner(4, 64, 128, 20, 20)) + 4 * 20 * 20 * 64 * 2 + 128 * 64 * 4
+    # the least workspace the call accepts is the fp32-ALU kernel's
+    assert 256 <= ac.ac_workspace_bytes_min(d) < ac.ac_workspace_bytes(d)
+    # more than 256 columns, other dtypes or layouts, C_out not a multiple of 64: not taken
+    for d in (ac.ConvDesc(4, 32, 64, 20, 20, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"),
+              ac.ConvDesc(4, 3, 64, 20, 20, 3, 3, (1, 1), (1, 1), 2, "f32", "nhwc"),
+              ac.ConvDesc(4, 3, 64, 20, 20, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
+              ac.ConvDesc(4, 3, 40, 20, 20, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")):
+        assert ac.ac_wgrad_plan_info(d)["tensor_core"] != 5

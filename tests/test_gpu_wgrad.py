@@ -407,3 +407,44 @@ def test_collapsed_form_full_size_and_refusals():
         with pytest.raises(ac.AcError) as e:
             ac.ac_conv2d_wgrad_compressed_collapsed(bad, t, t, t, t, 4096)
         assert e.value.status == ac.api.AC_ERR_UNSUPPORTED
+
+
+# Few input channels (bf16 NHWC): the operand is gathered into a [positions][taps x channels] matrix
+# and the tensor-core kernel runs the equivalent 1x1 problem (plan code 5).
+FEW_CHANNELS = [
+    # N, Ci, Co, H, W, R, S, stride, pad, k
+    (2, 3, 64, 32, 32, 7, 7, 2, 3, 2),      # stem-like: stride = k, k | H: 49 taps collapse to 16 shifts
+    (2, 3, 64, 31, 29, 7, 7, 2, 3, 2),      # odd map: partial last blocks, one column per tap
+    (3, 3, 128, 20, 20, 3, 3, 1, 1, 2),     # stride 1 at k = 2: no collapse
+    (2, 5, 128, 20, 20, 5, 5, 2, 2, 4),     # stride does not reach k
+    (2, 4, 64, 24, 24, 5, 5, 4, 2, 2),      # stride = 2k: two pooled rows per output row
+    (2, 3, 64, 16, 16, 7, 7, 2, 3, 1),      # k = 1
+    (2, 16, 64, 12, 12, 3, 3, 1, 1, 2),     # 144 columns -> 192
+    (1, 1, 64, 9, 9, 3, 3, 1, 0, 3),        # one channel, k = 3, no padding
+    (2, 3, 64, 32, 32, 3, 5, 2, 1, 2),      # R != S, collapsed
+    (2, 7, 192, 8, 8, 1, 1, 1, 0, 2),       # pointwise
+]
+
+
+@pytest.mark.parametrize("case", FEW_CHANNELS)
+def test_few_input_channels_match_checker(case):
+    import paper_2409_11902_b200 as ac
+    d = D(*case, "bf16", "nhwc")
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 5
+    err, got, want = wgrad_error_full(d)
+    assert err <= 1e-4 <= TOL_DW["bf16"], err     # bf16 products are exact in fp32: summation order only
+
+
+def test_few_input_channels_small_workspace_and_full_size_stem():
+    import paper_2409_11902_b200 as ac
+    import oracle
+    from paper_2409_11902_b200 import synth
+    d = D(2, 3, 64, 32, 32, 7, 7, 2, 3, 2, "bf16", "nhwc")
+    z, dy = make_wgrad_inputs(d)
+    want = oracle.wgrad_compressed(synth.to_f64(z), synth.to_f64(dy), d.H, d.W, d.R, d.S, d.stride, d.pad, d.k)
+    for nbytes in (ac.ac_workspace_bytes_min(d), ac.ac_workspace_bytes(d)):
+        got = run_wgrad(d, z, dy, nbytes=nbytes)
+        assert float(np.linalg.norm(got - want) / np.linalg.norm(want)) <= 1e-4
+    # the ResNet stem at its own map size
+    err, _ = wgrad_error_sampled(D(8, 3, 64, 224, 224, 7, 7, 2, 3, 2, "bf16", "nhwc"), n_samples=256)
+    assert err <= 1e-4, err
