@@ -67,8 +67,9 @@ typedef struct {
  * Bytes of scratch with which ac_conv2d_wgrad_compressed runs this problem on
  * its fastest path: a small status block, the split-K partial sums of dW and,
  * for fp32 and/or NCHW inputs that go to the tensor cores, bf16 NHWC copies of
- * Z and dY (see ac_conv2d_wgrad_compressed). Pure host code. Returns 0 for an
- * invalid descriptor.
+ * Z and dY, or, for layers with few input channels, the gathered operand matrix
+ * (see ac_conv2d_wgrad_compressed). Pure host code. Returns 0 for an invalid
+ * descriptor.
  */
 size_t ac_workspace_bytes(const ac_conv_desc *desc);
 
@@ -138,9 +139,15 @@ ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z
  * dropped); the split copies of Z and dY live in the workspace, which is why
  * ac_workspace_bytes is then about 3 x (|Z| + |dY|) x 4 bytes larger. NCHW
  * inputs that the tensor-core kernel takes once transposed are copied to NHWC
- * bf16 in the workspace in the same pass. All other fp32 or NCHW problems, and
- * calls whose workspace is smaller than ac_workspace_bytes but at least
- * ac_workspace_bytes_min, use fp32 FMA on the operands as they are.
+ * bf16 in the workspace in the same pass. bf16 NHWC layers with fewer than 64
+ * input channels (a network's first convolution) have the values every output
+ * position reads gathered into a [N*H_o*W_o][taps x C_in] bf16 matrix in the
+ * workspace (at most 256 columns, padded to a multiple of 64; taps that read
+ * the same element of Z for every position share one column) and run as the
+ * equivalent 1x1 problem on the tensor cores. All other problems, and calls
+ * whose workspace is smaller than ac_workspace_bytes but at least
+ * ac_workspace_bytes_min, use fp32 FMA (or the slower tensor-core kernel) on
+ * the operands as they are.
  *
  *   z          in : as produced by ac_compress.
  *   dy         in : [N,C_out,H_o,W_o], desc->layout / desc->dtype.
@@ -260,7 +267,13 @@ ac_status ac_conv2d_wgrad_compressed_static(const ac_conv_desc *desc, const void
  * reports and tests). Returns AC_ERR_INVALID_ARG for an invalid descriptor.
  */
 typedef struct {
-    int32_t tensor_core;     /* 4: as 3, but as two launches whose results are added: the five small
+    int32_t tensor_core;     /* 5: bf16 NHWC with fewer than 64 input channels (a 3-channel stem): the
+                                inflated, zero-padded values every output position reads are gathered
+                                into a [positions][taps x C_in] matrix in the workspace (one column
+                                per distinct shift of Z instead of per tap when both strides are
+                                multiples of k and k divides H and W), then as 2 on the equivalent
+                                1x1 problem over the output map (described by the other fields),
+                                4: as 3, but as two launches whose results are added: the five small
                                 partial products (five times the images; described by the other
                                 fields), then the leading one, 3: fp32 and/or NCHW inputs staged
                                 as bf16 NHWC terms in the workspace (fp32: six partial products =

@@ -201,63 +201,74 @@ permute_dw_kernel(const float* __restrict__ src, float* __restrict__ dst, int Ci
 // ---- few input channels: gathered operand ------------------------------------------------------
 struct GatherParams {
     int Ci, H, W, Hp, Wp, Ho, Wo, k;
+    int kshift;         // log2 k if k is a power of two, else -1
     int sh, sw, ph, pw;
     int collapsed;      // 1: one column per distinct Z shift (u, v); 0: one per tap (r, s)
     int mh, mw;         // collapsed: Z rows / columns per output row / column (s_h / k, s_w / k)
     int u0, v0;         // collapsed: first shift
-    int nb;             // shifts (collapsed) or taps per row of shifts / taps: nV or S
+    int na, nb;         // rows and columns of shifts (collapsed: nU, nV) or taps (R, S)
     int cols, Mp;       // valid columns (shifts or taps, times C_in), row length of G (multiple of 64)
-    long long groups;   // positions * Mp / 8
+    int rows;           // N * H_o output rows
+    int rows_per_block;
 };
 
-// G[position][column], eight columns (one 16-byte vector) per thread. Z is read element by element
-// (it is k^2 times smaller than what is written and stays in L2); consecutive threads write
-// consecutive vectors.
+// G[position][column], eight columns (one 16-byte vector) per thread, a block per `rows_per_block`
+// output rows. Z is read element by element (it is k^2 times smaller than what is written and stays
+// in L2); consecutive threads write consecutive vectors. Positions all of whose taps fall inside
+// the map (most of them) skip the bounds checks.
 __global__ void __launch_bounds__(256)
 gather_kernel(const unsigned short* __restrict__ z, uint4* __restrict__ g, const GatherParams p) {
-    __shared__ int tab[256];    // column -> a | b << 8 | channel << 16, or -1 behind the last column
+    __shared__ int tab_ab[256];     // column -> a | b << 8, or -1 behind the last column
+    __shared__ int tab_off[256];    // column -> offset in Z elements from the position's first element
     for (int j = threadIdx.x; j < p.Mp; j += 256) {
-        int e = -1;
+        int e = -1, off = 0;
         if (j < p.cols) {
             const int t = j / p.Ci, ci = j - t * p.Ci, a = t / p.nb, b = t - a * p.nb;
-            e = a | (b << 8) | (ci << 16);
+            e = a | (b << 8);
+            off = p.collapsed ? (a * p.Wp + b) * p.Ci + ci : ci;
         }
-        tab[j] = e;
+        tab_ab[j] = e;
+        tab_off[j] = off;
     }
     __syncthreads();
-    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
-    if (idx >= p.groups) return;
-    const int G = p.Mp / 8;
-    const long long pos = idx / G;
-    const int j0 = (int)(idx - pos * G) * 8;
-    const int wo = (int)(pos % p.Wo);
-    const long long t1 = pos / p.Wo;
-    const int ho = (int)(t1 % p.Ho);
-    const long long n = t1 / p.Ho;
-    const unsigned short* zn = z + n * p.Hp * p.Wp * p.Ci;
-    const int rb = p.collapsed ? ho * p.mh + p.u0 : ho * p.sh - p.ph;
-    const int cb = p.collapsed ? wo * p.mw + p.v0 : wo * p.sw - p.pw;
-    unsigned short v[8];
+    const int G = p.Mp / 8, per_row = p.Wo * G;
+    const int row0 = blockIdx.x * p.rows_per_block;
+    const int nrows = min(p.rows_per_block, p.rows - row0);
+    for (int v = threadIdx.x; v < nrows * per_row; v += 256) {
+        const int r = v / per_row, rem = v - r * per_row, wo = rem / G, j0 = (rem - wo * G) * 8;
+        const int row = row0 + r, n = row / p.Ho, ho = row - n * p.Ho;
+        const unsigned short* zn = z + (long long)n * p.Hp * p.Wp * p.Ci;
+        const int rb = p.collapsed ? ho * p.mh + p.u0 : ho * p.sh - p.ph;
+        const int cb = p.collapsed ? wo * p.mw + p.v0 : wo * p.sw - p.pw;
+        unsigned short val[8];
+        if (p.collapsed) {
+            const unsigned short* zb = zn + ((long long)rb * p.Wp + cb) * p.Ci;
+            if (rb >= 0 && rb + p.na <= p.Hp && cb >= 0 && cb + p.nb <= p.Wp) {
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-        const int e = tab[j0 + q];
-        unsigned short val = 0;
-        if (e >= 0) {
-            int zr = rb + (e & 255), zc = cb + ((e >> 8) & 255);
-            bool in;
-            if (p.collapsed) {
-                in = zr >= 0 && zr < p.Hp && zc >= 0 && zc < p.Wp;
+                for (int q = 0; q < 8; ++q) val[q] = tab_ab[j0 + q] >= 0 ? __ldg(zb + tab_off[j0 + q]) : 0;
             } else {
-                in = zr >= 0 && zr < p.H && zc >= 0 && zc < p.W;      // coordinates of the inflated map
-                zr /= p.k;
-                zc /= p.k;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int e = tab_ab[j0 + q];
+                    const bool in = e >= 0 && (unsigned)(rb + (e & 255)) < (unsigned)p.Hp &&
+                                    (unsigned)(cb + (e >> 8)) < (unsigned)p.Wp;
+                    val[q] = in ? __ldg(zb + tab_off[j0 + q]) : 0;
+                }
             }
-            if (in) val = __ldg(zn + ((long long)zr * p.Wp + zc) * p.Ci + (e >> 16));
+        } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int e = tab_ab[j0 + q];
+                int x = rb + (e & 255), y = cb + (e >> 8);      // coordinates of the inflated map
+                const bool in = e >= 0 && (unsigned)x < (unsigned)p.H && (unsigned)y < (unsigned)p.W;
+                if (p.kshift >= 0) { x >>= p.kshift; y >>= p.kshift; } else { x /= p.k; y /= p.k; }
+                val[q] = in ? __ldg(zn + ((long long)x * p.Wp + y) * p.Ci + tab_off[j0 + q]) : 0;
+            }
         }
-        v[q] = val;
+        g[((long long)row * p.Wo + wo) * G + (j0 >> 3)] =
+            make_uint4(val[0] | (uint32_t)val[1] << 16, val[2] | (uint32_t)val[3] << 16,
+                       val[4] | (uint32_t)val[5] << 16, val[6] | (uint32_t)val[7] << 16);
     }
-    g[idx] = make_uint4(v[0] | (uint32_t)v[1] << 16, v[2] | (uint32_t)v[3] << 16, v[4] | (uint32_t)v[5] << 16,
-                        v[6] | (uint32_t)v[7] << 16);
 }
 
 // dW[co][r][s][ci] = dW'[co][column of (r, s, ci)]
@@ -292,22 +303,27 @@ GatherGeom gather_geom(const Dims& d) {
     p.Ci = d.Ci; p.H = d.H; p.W = d.W; p.Hp = d.Hp; p.Wp = d.Wp; p.Ho = d.Ho; p.Wo = d.Wo; p.k = d.k;
     p.sh = d.sh; p.sw = d.sw; p.ph = d.ph; p.pw = d.pw;
     p.collapsed = d.k > 1 && d.sh % d.k == 0 && d.sw % d.k == 0 && d.H % d.k == 0 && d.W % d.k == 0;
-    int na = d.R;
+    p.kshift = -1;
+    for (int b = 0; b < 30; ++b) if (d.k == (1 << b)) p.kshift = b;
+    p.na = d.R;
     p.nb = d.S;
     if (p.collapsed) {
         p.mh = d.sh / d.k; p.mw = d.sw / d.k;
         p.u0 = floor_div_i(-d.ph, d.k); p.v0 = floor_div_i(-d.pw, d.k);
-        na = floor_div_i(d.R - 1 - d.ph, d.k) - p.u0 + 1;
+        p.na = floor_div_i(d.R - 1 - d.ph, d.k) - p.u0 + 1;
         p.nb = floor_div_i(d.S - 1 - d.pw, d.k) - p.v0 + 1;
     }
-    const long long cols = (long long)na * p.nb * d.Ci;
+    const long long cols = (long long)p.na * p.nb * d.Ci;
     if (cols > 256) return g;
     p.cols = (int)cols;
     p.Mp = (p.cols + 63) / 64 * 64;
-    const long long positions = d.K();
-    if (positions * p.Mp >= (1ll << 40)) return g;
-    p.groups = positions * (p.Mp / 8);
-    if ((p.groups + 255) / 256 >= (1ll << 31)) return g;
+    if (d.K() * p.Mp >= (1ll << 40) || (long long)d.N * d.Ho >= (1ll << 31)) return g;
+    if ((long long)d.Hp * d.Wp * d.Ci >= (1ll << 31)) return g;      // offsets within one image are 32-bit
+    p.rows = d.N * d.Ho;
+    // about 1024 vectors (four per thread) per block, whole output rows
+    const long long per_row = (long long)d.Wo * (p.Mp / 8);
+    if (per_row >= (1ll << 24)) return g;
+    p.rows_per_block = (int)(per_row >= 1024 ? 1 : (1024 + per_row - 1) / per_row);
     Dims in = d;
     in.Ci = p.Mp;
     in.H = in.Hp = d.Ho;
@@ -508,7 +524,7 @@ ac_status launch_wgrad_gather(const Dims& d, const WgradPlan& pl, const void* z,
     char* ws = static_cast<char*>(workspace);
     uint4* gm = reinterpret_cast<uint4*>(ws + pl.st_off_z);
     float* dw_cols = reinterpret_cast<float*>(ws + pl.st_off_dw);
-    gather_kernel<<<(unsigned)((g.p.groups + 255) / 256), 256, 0, stream>>>(
+    gather_kernel<<<(unsigned)((g.p.rows + g.p.rows_per_block - 1) / g.p.rows_per_block), 256, 0, stream>>>(
         static_cast<const unsigned short*>(z), gm, g.p);
     AC_CUDA_TRY(cudaGetLastError());
     const ac_status st = launch_wgrad_tc2(g.in, pl, gm, dy, dw_cols, workspace, stream);
