@@ -271,6 +271,65 @@ gather_kernel(const unsigned short* __restrict__ z, uint4* __restrict__ g, const
     }
 }
 
+// The same matrix for the collapsed form, built from shared memory: the `na` rows of Z that one output
+// row reads are copied in once (coalesced, zeros where the row or column lies outside Z), and every
+// 16-byte vector of G is assembled from them, so that global memory sees Z once per output row and
+// the eight element reads per vector are shared-memory reads.
+constexpr int kGatherRowsSmemMax = 40 * 1024;
+constexpr int kGatherRowGroup = 4;      // output rows built per round from one set of Z rows
+
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const unsigned short* __restrict__ z, uint4* __restrict__ g, const GatherParams p) {
+    extern __shared__ unsigned short zs[];      // [(kGatherRowGroup - 1) * mh + na][span]
+    const int span = ((p.Wo - 1) * p.mw + p.nb) * p.Ci, row_elems = p.Wp * p.Ci;
+    // The block has a multiple of G = Mp / 8 threads, so a thread builds the same eight columns for
+    // every position it visits: their offsets in zs (from the position's first element) stay in registers.
+    const int G = p.Mp / 8, T = blockDim.x, wo_step = T / G;
+    const int wo_first = threadIdx.x / G, j0 = (threadIdx.x - wo_first * G) * 8;
+    int off[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int j = j0 + q;
+        off[q] = -1;
+        if (j < p.cols) {
+            const int t = j / p.Ci, ci = j - t * p.Ci, a = t / p.nb, b = t - a * p.nb;
+            off[q] = a * span + b * p.Ci + ci;
+        }
+    }
+    const int row0 = blockIdx.x * p.rows_per_block;
+    const int row1 = min(row0 + p.rows_per_block, p.rows);
+    for (int row = row0; row < row1;) {
+        // up to kGatherRowGroup output rows of one image per round: they share most of their Z rows
+        const int n = row / p.Ho, ho = row - n * p.Ho, rb = ho * p.mh + p.u0;
+        const int ng = min(min(kGatherRowGroup, row1 - row), p.Ho - ho);
+        const int nz = (ng - 1) * p.mh + p.na;
+        if (row > row0) __syncthreads();      // the rows before these have been read
+        for (int a = 0; a < nz; ++a) {
+            const int zr = rb + a;
+            const bool row_in = zr >= 0 && zr < p.Hp;
+            const unsigned short* src = z + ((long long)n * p.Hp + zr) * row_elems;
+            for (int x = threadIdx.x; x < span; x += T) {
+                const int sx = x + p.v0 * p.Ci;      // element of the Z row
+                zs[a * span + x] = row_in && sx >= 0 && sx < row_elems ? __ldg(src + sx) : (unsigned short)0;
+            }
+        }
+        __syncthreads();
+        for (int r = 0; r < ng; ++r) {
+            uint4* grow = g + (long long)(row + r) * p.Wo * G + (j0 >> 3);
+            const unsigned short* zrow = zs + r * p.mh * span;
+            for (int wo = wo_first; wo < p.Wo; wo += wo_step) {
+                const unsigned short* zb = zrow + wo * p.mw * p.Ci;
+                unsigned short val[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) val[q] = off[q] >= 0 ? zb[off[q]] : (unsigned short)0;
+                grow[wo * G] = make_uint4(val[0] | (uint32_t)val[1] << 16, val[2] | (uint32_t)val[3] << 16,
+                                          val[4] | (uint32_t)val[5] << 16, val[6] | (uint32_t)val[7] << 16);
+            }
+        }
+        row += ng;
+    }
+}
+
 // dW[co][r][s][ci] = dW'[co][column of (r, s, ci)]
 __global__ void __launch_bounds__(256)
 scatter_columns_kernel(const float* __restrict__ src, float* __restrict__ dw, const GatherParams p, int R, int S,
@@ -524,13 +583,28 @@ ac_status launch_wgrad_gather(const Dims& d, const WgradPlan& pl, const void* z,
     char* ws = static_cast<char*>(workspace);
     uint4* gm = reinterpret_cast<uint4*>(ws + pl.st_off_z);
     float* dw_cols = reinterpret_cast<float*>(ws + pl.st_off_dw);
-    gather_kernel<<<(unsigned)((g.p.rows + g.p.rows_per_block - 1) / g.p.rows_per_block), 256, 0, stream>>>(
-        static_cast<const unsigned short*>(z), gm, g.p);
+    GatherParams gp = g.p;
+    const long long rows_smem =
+        2ll * ((kGatherRowGroup - 1) * gp.mh + gp.na) * (((long long)gp.Wo - 1) * gp.mw + gp.nb) * gp.Ci;
+    if (gp.collapsed && rows_smem <= kGatherRowsSmemMax) {
+        // a thread works out its eight column offsets once per block: give a block about 64 vectors per
+        // thread, as long as that leaves four blocks for every SM
+        const long long per_row = (long long)gp.Wo * (gp.Mp / 8);
+        long long rpb = (16384 + per_row - 1) / per_row;
+        if (rpb > gp.rows / (4 * kNumSMs)) rpb = gp.rows / (4 * kNumSMs);
+        if (rpb > gp.rows_per_block) gp.rows_per_block = (int)rpb;
+        const unsigned blocks = (unsigned)((gp.rows + gp.rows_per_block - 1) / gp.rows_per_block);
+        gather_rows_kernel<<<blocks, 256 / (gp.Mp / 8) * (gp.Mp / 8), (size_t)rows_smem, stream>>>(
+            static_cast<const unsigned short*>(z), gm, gp);
+    } else {
+        const unsigned blocks = (unsigned)((gp.rows + gp.rows_per_block - 1) / gp.rows_per_block);
+        gather_kernel<<<blocks, 256, 0, stream>>>(static_cast<const unsigned short*>(z), gm, gp);
+    }
     AC_CUDA_TRY(cudaGetLastError());
     const ac_status st = launch_wgrad_tc2(g.in, pl, gm, dy, dw_cols, workspace, stream);
     if (st != AC_OK) return st;
     const long long total = d.dw_elems();
-    scatter_columns_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(dw_cols, dw, g.p, d.R, d.S, total);
+    scatter_columns_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(dw_cols, dw, gp, d.R, d.S, total);
     AC_CUDA_TRY(cudaGetLastError());
     return AC_OK;
 }

@@ -22,6 +22,9 @@ LAYERS = {
     "128ch_64x64": (128, 128, 64, 64, 3, 3, 1, 1),
     "128ch_56x56_s2": (128, 128, 56, 56, 3, 3, 2, 1),
     "256to64_1x1_56x56": (256, 64, 56, 56, 1, 1, 1, 0),
+    "256to1024_1x1_14x14": (256, 1024, 14, 14, 1, 1, 1, 0),
+    "1024to256_1x1_14x14": (1024, 256, 14, 14, 1, 1, 1, 0),
+    "3to64_7x7_s2_224x224": (3, 64, 224, 224, 7, 7, 2, 3),
 }
 
 

@@ -27,6 +27,12 @@ SHAPES = [
     (2, 24, 9, 15),      # odd H and W, C a multiple of 8
     (1, 3, 17, 23),      # stem-like: C not a multiple of the vector width
     (1, 5, 1, 1),        # degenerate map
+    # NHWC with C not a multiple of the vector width but W * C one
+    (2, 3, 32, 32),
+    (3, 3, 15, 24),      # odd H: a partial last row of blocks
+    (2, 4, 9, 14),       # partial blocks in both directions at k = 4
+    (1, 12, 7, 10),
+    (2, 3, 224, 224),    # the ResNet stem's input
 ]
 
 
@@ -43,7 +49,8 @@ def test_compress_matches_checker(shape, k, dtype, layout):
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("k", [1, 2, 4, 8])
 @pytest.mark.parametrize("inplace", [False, True])
-@pytest.mark.parametrize("shape", [(3, 64, 56, 56), (2, 512, 7, 7), (1, 3, 17, 23), (2, 32, 16, 64)])
+@pytest.mark.parametrize("shape", [(3, 64, 56, 56), (2, 512, 7, 7), (1, 3, 17, 23), (2, 32, 16, 64),
+                                   (2, 3, 32, 32), (3, 3, 15, 24), (2, 4, 9, 14)])
 def test_fused_relu_compress(shape, inplace, k, dtype, layout):
     err, _, _ = run_compress(desc(*shape, k, dtype, layout), fused_relu=True, inplace=inplace)
     assert err <= TOL_Z[dtype], err
