@@ -40,6 +40,27 @@ BOTTLENECK = [(256, 64, 56, 1, 1, 0, 1), (64, 64, 56, 3, 1, 1, 1), (64, 256, 56,
 RESNET18_STACK = [(64, 64, 56, 3, 1, 1, 1), (128, 128, 28, 3, 1, 1, 1), (256, 256, 14, 3, 1, 1, 1),
                   (512, 512, 8, 3, 1, 1, 1), (512, 512, 7, 3, 1, 1, 1)]
 WORKLOADS = {"resnet50": (RESNET50, 256), "bottleneck": (BOTTLENECK, 128), "resnet18_stack": (RESNET18_STACK, 64)}
+# ResNet-50 convolutions whose input another convolution reads too (the first block of a stage feeds
+# both conv1 and the downsample projection): that tensor is saved, and compressed, once.
+RESNET50_SHARED_INPUT = {(64, 256, 56, 1, 1): 1, (256, 512, 56, 1, 2): 1, (512, 1024, 28, 1, 2): 1,
+                         (1024, 2048, 14, 1, 2): 1}
+
+
+def saved_state_model(layers, N, k, elt, shared):
+    """Bytes a training step keeps for backward in a conv -> batch-norm -> ReLU network, by accounting
+    (no step is run): A = the distinct conv inputs (each is also the output its ReLU keeps), B = the
+    conv outputs (what each batch-norm keeps). The paper's scheme stores A / k^2 instead of A; a ReLU
+    that feeds only compressed convolutions then needs one bit per element for its own backward."""
+    A = B = Az = 0
+    for ci, co, H, R, st, pd, cnt in layers:
+        distinct = cnt - shared.get((ci, co, H, R, st), 0)
+        Ho = (H + 2 * pd - R) // st + 1
+        Hp = -(-H // k)
+        A += distinct * N * ci * H * H * elt
+        Az += distinct * N * ci * Hp * Hp * elt
+        B += cnt * N * co * Ho * Ho * elt
+    mask = A // (8 * elt)
+    return A, Az, B, mask
 
 
 def load_peaks(path):
@@ -139,6 +160,14 @@ def main():
           f"({tot['cb'] / tot['tc'] / 1e3 / hbm:.2f} of HBM); wgrad {tot['tw']:.0f} us = {tot['fl'] / tot['tw'] / 1e6:.0f} TFLOP/s "
           f"dense-equivalent ({tot['bound_us'] / tot['tw']:.2f} of the per-layer bounds, "
           f"{tot['fl'] / tot['tw'] / 1e6 / tens:.2f} of the tensor peak).")
+    if a.workload == "resnet50":
+        A, Az, B, mask = saved_state_model(layers, N, a.k, elt, RESNET50_SHARED_INPUT)
+        m = 2.0 ** 20
+        print(f"\nSaved-for-backward state by accounting (conv -> batch-norm -> ReLU; no training step is run): distinct conv "
+              f"inputs {A / m:.0f} MiB + conv outputs kept by batch-norm {B / m:.0f} MiB = {(A + B) / m:.0f} MiB. With Z in "
+              f"place of the conv inputs: {Az / m:.0f} + {B / m:.0f} = {(Az + B) / m:.0f} MiB (-{100 * (A - Az) / (A + B):.1f} %); "
+              f"with one mask bit per element for the ReLUs' own backward: {(Az + mask + B) / m:.0f} MiB "
+              f"(-{100 * (A - Az - mask) / (A + B):.1f} %).")
 
 
 if __name__ == "__main__":

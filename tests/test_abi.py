@@ -209,3 +209,29 @@ def test_few_input_channels_are_gathered_for_the_tensor_cores(ac):
               ac.ConvDesc(4, 3, 64, 20, 20, 3, 3, (1, 1), (1, 1), 2, "bf16", "nchw"),
               ac.ConvDesc(4, 3, 40, 20, 20, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")):
         assert ac.ac_wgrad_plan_info(d)["tensor_core"] != 5
+
+
+def test_layer_report_tables_match_the_network():
+    """The report tool's ResNet-50 layer table and saved-state accounting against an independent
+    walk over the network (bottleneck blocks, stride on the 3x3, 224 x 224 images, batch 256, bf16)."""
+    from paper_2409_11902_b200 import layer_report as lr
+    assert sum(l[-1] for l in lr.RESNET50) == 53 and len(lr.RESNET50) == 23
+    inputs, outputs, flops = [(3, 224)], [(64, 112)], 2 * 112 * 112 * 64 * 3 * 49
+    for cin, width, cout, H, blocks, stride in [(64, 64, 256, 56, 3, 1), (256, 128, 512, 56, 4, 2),
+                                                (512, 256, 1024, 28, 6, 2), (1024, 512, 2048, 14, 3, 2)]:
+        for b in range(blocks):
+            h_in = H if b == 0 else H // stride
+            h_out = H // stride
+            c_in = cin if b == 0 else cout
+            inputs += [(c_in, h_in), (width, h_in), (width, h_out)]
+            outputs += [(width, h_in), (width, h_out), (cout, h_out)] + ([(cout, h_out)] if b == 0 else [])
+            flops += 2 * (h_in * h_in * width * c_in + h_out * h_out * width * width * 9 + h_out * h_out * cout * width
+                          + (h_out * h_out * cout * c_in if b == 0 else 0))
+    A, Az, B, mask = lr.saved_state_model(lr.RESNET50, 256, 2, 2, lr.RESNET50_SHARED_INPUT)
+    assert A == sum(256 * c * h * h * 2 for c, h in inputs)
+    assert Az == sum(256 * c * (-(-h // 2)) ** 2 * 2 for c, h in inputs)
+    assert B == sum(256 * c * h * h * 2 for c, h in outputs)
+    assert mask == A // 16
+    table_flops = sum(cnt * 2 * ((H + 2 * pd - R) // st + 1) ** 2 * co * ci * R * R
+                      for ci, co, H, R, st, pd, cnt in lr.RESNET50)
+    assert table_flops == flops
