@@ -71,6 +71,7 @@ struct Tc2Params {
     // 0. A (class, tap) pair whose x falls in that second range at the last Z row is served from a
     // copy of the tile fetched through a tensor map that ends one row (column) earlier.
     int nvar, var_slot[4], rho_h, rho_w;   // variants in use, variant -> position in the slot, H % k, W % k
+    int Hp, Wp, Ho, Wo;                    // pooled and output map sizes (which pairs need a variant)
     long long dw_elems;
     // Paired mode (64 input channels): one accumulator tile holds TWO taps, rows 0-63
     // tap A and rows 64-127 tap B, because the input tile is kept in up to three copies
@@ -91,6 +92,23 @@ struct Tc2Params {
     int chunk_kt;
     long long slice_elems;   // floats of one K-slice of the partial tensor
 };
+
+// Whether outputs of class row `a` (ho = a, a + k/s, ...) read, through tap row r, one of the rows
+// x in [H, k*Hp) that the convolution pads with zeros but the partial last row of Z covers. Every x
+// this pair reads, x = s*ho - pad + r, has the same remainder rem = (s*a - pad + r) mod k, so the one
+// candidate is x = k*(Hp-1) + rem with rem >= rho = H mod k; it is read only if the ho it belongs
+// to is an output row (a 1x1 layer without padding never reads beyond H, whatever the map size).
+// The same function serves columns.
+__host__ __device__ inline bool reads_padding_in_partial_block(int s, int a, int pad, int r, int k, int Hp,
+                                                               int rho, int Ho) {
+    if (rho == 0) return false;
+    const int c = s * a - pad + r;
+    const int rem = c - floor_div_i(c, k) * k;
+    if (rem < rho) return false;
+    const int num = k * (Hp - 1) + rem + pad - r;      // s * ho of the candidate
+    if (num < 0 || num % s != 0) return false;
+    return num / s < Ho;
+}
 
 // Distinct Z shifts of output class `cls`: rows u0 .. u0+nU-1, columns v0 .. v0+nV-1
 // (u = floor((s_h*a - p_h + r) / k) is non-decreasing in r with steps of 0 or 1).
@@ -332,9 +350,8 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 const int vv = floor_div_i(p.sw * b - p.pw + sx, p.k) - p.vmin;
                 // which copy of the tile: the one without the partial last row / column of Z if this
                 // (class, tap) reaches past H / W there
-                const int ch_ = p.sh * a - p.ph + r, cw_ = p.sw * b - p.pw + sx;
-                const int rh = ch_ - floor_div_i(ch_, p.k) * p.k, rw = cw_ - floor_div_i(cw_, p.k) * p.k;
-                const int var = ((p.rho_h > 0 && rh >= p.rho_h) ? 2 : 0) + ((p.rho_w > 0 && rw >= p.rho_w) ? 1 : 0);
+                const int var = (reads_padding_in_partial_block(p.sh, a, p.ph, r, p.k, p.Hp, p.rho_h, p.Ho) ? 2 : 0) +
+                                (reads_padding_in_partial_block(p.sw, b, p.pw, sx, p.k, p.Wp, p.rho_w, p.Wo) ? 1 : 0);
                 off = (uint32_t)(p.var_slot[var] * p.chunksA + cl * (p.CB / 64)) * p.a_chunk_bytes +
                       (uint32_t)(uu * p.Wzq + vv) * 128u;
             }
@@ -753,14 +770,14 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     int chunksA = up.CB == 128 ? 2 * up.cibs_per_group : up.cibs_per_group + 1;
     // which copies of the Z tile are needed (see Tc2Params::nvar)
     p.rho_h = d.H % d.k; p.rho_w = d.W % d.k;
+    p.Hp = d.Hp; p.Wp = d.Wp; p.Ho = d.Ho; p.Wo = d.Wo;
     bool var_used[4] = {false, false, false, false};
     for (int a = 0; a < p.c_h; ++a)
         for (int r = 0; r < d.R; ++r)
             for (int b = 0; b < p.c_w; ++b)
                 for (int s_ = 0; s_ < d.S; ++s_) {
-                    const int ch_ = d.sh * a - d.ph + r, cw_ = d.sw * b - d.pw + s_;
-                    const int rh = ch_ - floor_div_i(ch_, d.k) * d.k, rw = cw_ - floor_div_i(cw_, d.k) * d.k;
-                    var_used[((p.rho_h > 0 && rh >= p.rho_h) ? 2 : 0) + ((p.rho_w > 0 && rw >= p.rho_w) ? 1 : 0)] = true;
+                    var_used[(reads_padding_in_partial_block(d.sh, a, d.ph, r, d.k, d.Hp, p.rho_h, d.Ho) ? 2 : 0) +
+                             (reads_padding_in_partial_block(d.sw, b, d.pw, s_, d.k, d.Wp, p.rho_w, d.Wo) ? 1 : 0)] = true;
                 }
     p.nvar = 0;
     for (int v = 0; v < 4; ++v) p.var_slot[v] = var_used[v] ? p.nvar++ : -1;

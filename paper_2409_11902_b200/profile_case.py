@@ -24,6 +24,8 @@ LAYERS = {
     "256to64_1x1_56x56": (256, 64, 56, 56, 1, 1, 1, 0),
     "256to1024_1x1_14x14": (256, 1024, 14, 14, 1, 1, 1, 0),
     "1024to256_1x1_14x14": (1024, 256, 14, 14, 1, 1, 1, 0),
+    "1024to2048_1x1_s2_14x14": (1024, 2048, 14, 14, 1, 1, 2, 0),
+    "512to2048_1x1_7x7": (512, 2048, 7, 7, 1, 1, 1, 0),
     "3to64_7x7_s2_224x224": (3, 64, 224, 224, 7, 7, 2, 3),
 }
 

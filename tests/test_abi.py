@@ -147,6 +147,11 @@ def test_plan_info_respects_hardware_limits(ac):
     # a map that k does not divide (partial pooling blocks) is still taken by the TMA-fed kernel
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 512, 512, 7, 7, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
     assert i["tensor_core"] == 2
+    # ... and a 1x1 layer without padding never reads the padding rows inside the partial last block,
+    # so it needs no second copy of the tile: same tiles as on the 8x8 map
+    i7, i8 = (ac.ac_wgrad_plan_info(ac.ConvDesc(256, 512, 2048, h, h, 1, 1, (1, 1), (0, 0), 2, "bf16", "nhwc"))
+              for h in (7, 8))
+    assert all(i7[f] == i8[f] for f in ("k_tile", "stages", "smem_bytes", "a_cells", "row_pitch", "ctas"))
     # a stride that does not divide k goes to the producer-fed tensor-core kernel
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 28, 28, 3, 3, (2, 2), (1, 1), 1, "bf16", "nhwc"))
     assert i["tensor_core"] == 1

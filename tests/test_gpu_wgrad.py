@@ -39,6 +39,12 @@ SMALL = [
     (2, 24, 40, 10, 10, 5, 3, 1, 2, 2),     # channels not multiples of 64, R != S
     (1, 8, 8, 4, 4, 3, 3, 1, 1, 2),         # tiny
     (1, 64, 64, 1, 1, 1, 1, 1, 0, 2),       # degenerate map
+    # odd maps whose outputs never read the padding rows inside the partial last block (no padding):
+    # served from the one full copy of the Z tile
+    (3, 128, 64, 7, 9, 1, 1, 1, 0, 2),
+    (2, 64, 128, 9, 7, 3, 3, 1, 0, 2),
+    (2, 64, 64, 10, 10, 1, 1, 1, 0, 4),
+    (2, 64, 64, 11, 11, 3, 3, 2, 0, 2),
 ]
 
 
