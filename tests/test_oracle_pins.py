@@ -232,6 +232,37 @@ def test_tap_collapse_stride2_k2():
     assert not np.array_equal(dw[:, :, 0, :], dw[:, :, 1, :])
 
 
+@pytest.mark.parametrize("R,stride,pad,k,H", [(7, 2, 3, 2, 12), (5, 4, 2, 2, 16), (3, 4, 1, 4, 16), (7, 2, 3, 2, 11)])
+def test_strides_that_are_multiples_of_k_read_one_shift_per_tap(R, stride, pad, k, H):
+    """When the stride is a multiple of k and k | H, output ho reads Z row ho*stride/k + floor((r - pad)/k)
+    through tap r, for every ho: dW[..., r, s] is the plain correlation of Z, shifted by that row and
+    column, with dY (written here as its own loop nest), and taps with equal shifts are equal. With a
+    partial last block (k does not divide H) the equality of such taps breaks at the padding edge."""
+    N, Ci, Co = 2, 2, 3
+    Hp = -(-H // k)
+    Ho = (H + 2 * pad - R) // stride + 1
+    z = RNG.standard_normal((N, Ci, Hp, Hp))
+    dy = RNG.standard_normal((N, Co, Ho, Ho))
+    dw = oracle.wgrad_compressed(z, dy, H, H, R, R, (stride, stride), (pad, pad), k)
+    shift = [(r - pad) // k for r in range(R)]           # Python's // floors
+    if H % k:
+        r0, r1 = R - 2, R - 1                             # same shift, but r1 reaches the padding row inside the block
+        assert shift[r0] == shift[r1] and not np.allclose(dw[:, :, r1, :], dw[:, :, r0, :])
+        return
+    m = stride // k
+    zpad = np.zeros((N, Ci, Hp + 2 * R + m * Ho, Hp + 2 * R + m * Ho))
+    zpad[:, :, R:R + Hp, R:R + Hp] = z
+    for r in range(R):
+        for s_ in range(R):
+            win = zpad[:, :, R + shift[r]:R + shift[r] + m * Ho:m, R + shift[s_]:R + shift[s_] + m * Ho:m]
+            want = np.einsum("nipq,nopq->oi", win, dy)
+            np.testing.assert_allclose(dw[:, :, r, s_], want, rtol=1e-12, atol=1e-13)
+    for r in range(1, R):
+        if shift[r] == shift[r - 1]:
+            assert np.array_equal(dw[:, :, r, :], dw[:, :, r - 1, :])
+            assert np.array_equal(dw[:, :, :, r], dw[:, :, :, r - 1])
+
+
 @pytest.mark.parametrize("k", [2, 4])
 def test_pointwise_conv_closed_form(k):
     """1x1, stride 1, k | H: dW[co,ci] = k^2 * sum Z * pool_k(dY)."""
