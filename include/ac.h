@@ -124,8 +124,8 @@ ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z
                                 void *mask, void *stream);
 
 /*
- * Weight gradient from the compressed activation (Section 4: inflate Z to the
- * original dimensions, then calculate the weight gradient normally; figure:
+ * Weight gradient from the compressed activation (Section 4: Z is expanded to
+ * X's shape and the ordinary weight gradient is taken of that; figure:
  * dL/dW ~ Z (*) dL/dY). With Xt[n,c,h,w] = Z[n,c,h/k,w/k] for 0<=h<H, 0<=w<W
  * and 0 elsewhere (the convolution's zero padding, applied after inflation):
  *
@@ -173,8 +173,8 @@ ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc *desc, const void *z,
 /*
  * The same weight gradient added to what dW holds (gradient accumulation over
  * micro-batches): dW <- beta * dW + (the result of ac_conv2d_wgrad_compressed).
- * The paper overwrites ("calculate the weight gradient normally", Section 4);
- * this is the usual framework convenience on top. The new gradient is formed
+ * Section 4 defines dW as a value that is assigned, not added to; accumulation
+ * is the usual framework convenience on top. The new gradient is formed
  * in the workspace by exactly the path ac_conv2d_wgrad_compressed would take
  * with `workspace_bytes - 4*|dW|` bytes (rounded down to 256), then one pass
  * combines it with dW, so the result is bitwise beta*dW + that gradient, in
@@ -249,8 +249,15 @@ ac_status ac_backward_step_host(const ac_conv_desc *desc, const void *x_host,
  *
  * Computes the same dW as ac_conv2d_wgrad_compressed (same arguments z, dy,
  * dw, same layouts, dW overwritten), always on the fp32-ALU kernel.
- *   - Problems whose split-K scratch would exceed AC_STATIC_SCRATCH_BYTES are
- *     refused with AC_ERR_WORKSPACE_TOO_SMALL before anything is launched.
+ *   - The sum over the N*H_o*W_o positions is cut into as many slices as the
+ *     array holds partial dW tensors for (256 bytes of it are the status
+ *     block), each slice one fp32 running sum per output. A slice may be up to
+ *     16384 positions long (the ordinary call stops at 2048, so this call's
+ *     fp32 rounding error can be a few times larger); a problem that would
+ *     need longer slices, because |dW| x 4 bytes x slices does not fit
+ *     AC_STATIC_SCRATCH_BYTES, is refused with AC_ERR_WORKSPACE_TOO_SMALL
+ *     before anything is launched. Problems of at most 16384 positions are
+ *     never refused (one slice goes straight to dW).
  *   - The first call on each device looks up the array's device address (the
  *     device must be current). Make that first call outside any stream capture.
  *   - All calls on a device share the one array, which still holds the last
@@ -301,9 +308,9 @@ typedef struct {
 ac_status ac_wgrad_plan_info(const ac_conv_desc *desc, ac_plan_info *info);
 
 /*
- * The same weight gradient with the repeated products taken out (the paper's remark that the
- * compressed form can "reduce the number of memory transactions" taken one step further; Section 4
- * defines only the result, which is unchanged). Inflation makes neighbouring taps read the same
+ * The same weight gradient with the repeated products taken out (Section 4 notes that a fused
+ * operator on the compressed form could also cut memory traffic; this goes one step further and
+ * cuts arithmetic. Section 4 defines only the result, which is unchanged). Inflation makes neighbouring taps read the same
  * pooled value: for the outputs of one class (ho mod k/s_h, wo mod k/s_w) every filter tap reads Z
  * at one of a few distinct shifts, and taps with the same shift form identical products. This call
  * accumulates one tile per (class, distinct shift) and adds each tile to all taps that map to it:

@@ -12,11 +12,11 @@
  *   pool      Z = average pooling of the layer INPUT X with non-overlapping
  *             k x k blocks that start at index (0,0) (figure: mu_00 is the
  *             mean of X_00, X_01, X_10, X_11).
- *   inflate   the stored Z is expanded "back to the original dimensions":
- *             every block mean stands for each element of its block.
- *   wgrad     the weight gradient is then calculated "normally" from the
- *             inflated tensor and the uncompressed output gradient:
- *             dL/dW ~ Z (*) dL/dY in the figure.
+ *   inflate   the stored Z is expanded to X's shape again: every block
+ *             mean stands for each element of its block.
+ *   wgrad     the ordinary weight gradient, taken of the inflated tensor
+ *             and the uncompressed output gradient: dL/dW ~ Z (*) dL/dY
+ *             in the figure.
  *
  * Readings where the paper is silent (all listed in the design notes):
  *   - H or W not divisible by k: the last block row/column is partial and is
@@ -128,8 +128,8 @@ void oracle_wgrad_dense(const double *x, const double *dy,
     }
 }
 
-/* Section 4, backward of a compressed layer: inflate the stored Z to X's
- * dimensions, then calculate the weight gradient normally.
+/* Section 4, backward of a compressed layer: the stored Z is inflated to X's
+ * shape and the ordinary weight gradient is taken of the result.
  * Returns 0, or -1 if the temporary cannot be allocated. */
 int oracle_wgrad_compressed(const double *z, const double *dy,
                             int64_t N, int64_t Ci, int64_t Co, int64_t H, int64_t W,

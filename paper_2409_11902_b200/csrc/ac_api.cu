@@ -36,7 +36,7 @@ ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o) {
 
 static inline long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
 
-WgradPlan plan_wgrad_simt(const Dims& d) {
+WgradPlan plan_wgrad_simt(const Dims& d, size_t max_partial_bytes) {
     WgradPlan p{};
     p.path = PATH_SIMT;
     const long long K = d.K();
@@ -49,7 +49,7 @@ WgradPlan plan_wgrad_simt(const Dims& d) {
     if (kps < 256) kps = 256;
     if (kps > 2048) kps = 2048;
     const long long dw_bytes = d.dw_elems() * 4;
-    long long max_splits = (256ll << 20) / dw_bytes;
+    long long max_splits = (long long)max_partial_bytes / dw_bytes;
     if (max_splits < 1) max_splits = 1;
     if (max_splits > 65535) max_splits = 65535;
     if (ceil_div(K, kps) > max_splits) kps = ceil_div(ceil_div(K, max_splits), 16) * 16;

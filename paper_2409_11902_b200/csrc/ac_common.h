@@ -56,7 +56,10 @@ struct WgradPlan {
 };
 
 WgradPlan plan_wgrad(const Dims& d);
-WgradPlan plan_wgrad_simt(const Dims& d);  // the fp32-ALU path's plan, whatever plan_wgrad picks
+// The fp32-ALU path's plan, whatever plan_wgrad picks. K-slices cover 256..2048 positions each unless
+// their partial sums would not fit `max_partial_bytes`; then there are fewer, longer slices (one
+// slice, written straight to dW, needs no scratch at all).
+WgradPlan plan_wgrad_simt(const Dims& d, size_t max_partial_bytes = (size_t)256 << 20);
 
 // ---- launchers (each enqueues on `stream`, returns AC_OK or AC_ERR_CUDA) -----
 ac_status launch_compress(const Dims& d, const void* x, void* z, void* y_out, cudaStream_t stream);

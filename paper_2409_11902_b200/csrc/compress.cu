@@ -125,9 +125,11 @@ __device__ __forceinline__ void store_mask(unsigned char* mask, long long elem_o
 // Grid: x covers the (q, channel vector) pairs of one pooled row, y = p, z = n,
 // so that no 64-bit division is needed. K > 0: pooling factor known at compile
 // time, all loads of up to four rows issued before the first use; K = 0: any k.
+// x is not __restrict__: the fused ReLU may run in place (y == x); a thread reads its own
+// elements before it writes them and no other thread touches them.
 template <typename T, int K, int MODE>   // MODE 0: pool only, 1: also store max(x,0), 2: also store the sign mask
 __global__ void __launch_bounds__(256)
-compress_nhwc_vec(const T* __restrict__ x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int CV,
+compress_nhwc_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int CV,
                   int k, int Hp, int Wp) {
     pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
     constexpr bool RELU = MODE != 0;
@@ -235,7 +237,7 @@ ac_status launch_nhwc_vec(const T* x, T* z, T* y, unsigned char* mask, long long
 // one warp shuffle when a block spans two lanes (fp32, k = 8).
 template <typename T, int K, int MODE, typename I>
 __global__ void __launch_bounds__(256)
-compress_nchw_vec(const T* __restrict__ x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int Hp,
+compress_nchw_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int Hp,
                   int Wp, long long total) {
     pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
     constexpr bool RELU = MODE != 0;

@@ -8,9 +8,10 @@
 // gathered into shared memory; Xt never exists in global memory.
 //
 // This path takes every dtype, layout, filter, stride, padding and k. It is
-// the only path for fp32 inputs (a single-pass TF32 tensor-core product cannot
-// meet the fp32 tolerance) and the fallback for shapes the tensor-core kernel
-// does not cover.
+// the fallback for shapes none of the tensor-core paths covers, for callers
+// whose workspace has no room for staged operand copies, and the kernel behind
+// the workspace-free entry point. The split-K reductions at the end of this
+// file serve the tensor-core kernels too.
 #include "ac_common.h"
 
 namespace ac {

@@ -22,6 +22,7 @@ namespace {
 static __device__ __align__(256) unsigned char g_static_scratch[AC_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
+constexpr long long kMaxStaticSlice = 16384;   // positions per K-slice (the ordinary plan stops at 2048)
 std::mutex g_mu;
 void* g_scratch_addr[kMaxDevices] = {};  // per device: device address of g_static_scratch
 
@@ -55,8 +56,11 @@ extern "C" ac_status ac_conv2d_wgrad_compressed_static(const ac_conv_desc* desc,
     if (st != AC_OK) return st;
     if (!z || !dy || !dw) return AC_ERR_INVALID_ARG;
     if (!aligned16(z) || !aligned16(dy) || !aligned16(dw)) return AC_ERR_MISALIGNED;
-    const WgradPlan p = plan_wgrad_simt(d);
-    if (p.bytes > (size_t)AC_STATIC_SCRATCH_BYTES) return AC_ERR_WORKSPACE_TOO_SMALL;
+    // As many K-slices as the fixed array holds, but no slice longer than kMaxStaticSlice positions:
+    // a slice is one fp32 running sum per output, and its rounding error grows with its length.
+    const WgradPlan p = plan_wgrad_simt(d, (size_t)AC_STATIC_SCRATCH_BYTES - kStatusBlockBytes);
+    if (p.bytes > (size_t)AC_STATIC_SCRATCH_BYTES || p.simt_k_per_split > kMaxStaticSlice)
+        return AC_ERR_WORKSPACE_TOO_SMALL;
     void* scratch = nullptr;
     st = scratch_for_current_device(&scratch);
     if (st != AC_OK) return st;

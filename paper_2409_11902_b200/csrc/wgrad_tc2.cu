@@ -13,16 +13,23 @@
 // and each (class, tap) pair is a shift (u,v) of Z. Zero padding falls out of
 // the tile bounds: x < 0 or x >= H  <=>  z < 0 or z >= H/k.
 //
-// So per K-tile (one band of class rows of one image):
-//   A operand: the Z halo tile, loaded by TMA, one 8-channel plane per copy,
-//              into the un-swizzled MN-major layout [plane][cell][8 channels];
-//              a (class, tap) pair only moves the descriptor's start address.
-//   B operand: for each class, the de-interleaved dY tile, loaded by TMA through
-//              a per-class tensor map (strides c_w*Co and c_h*Wo*Co), 128-byte
-//              swizzled, rows past the class's extent zero-filled by TMA.
+// Per K-tile (a band of class rows of one image, or several whole class images of a small map):
+//   A operand: the Z halo tile, one TMA copy per 64-channel chunk into the 128-byte-swizzled
+//              MN-major layout [cell][64 channels] (128 bytes per cell, as NHWC memory has
+//              them); a (class, tap) pair only moves the MMA descriptor's start address by
+//              whole cells. With partial pooling blocks (k does not divide H or W) up to four
+//              copies of the tile, fetched through tensor maps that end one row / column
+//              early, serve the taps that must read zero padding there. With 64 input
+//              channels up to three shifted copies let one M = 128 MMA compute two taps.
+//   B operand: for each class, the de-interleaved dY tile through a per-class tensor map
+//              (strides c_w*Co and c_h*Wo*Co; more than 16 classes: one map over dY walked
+//              with element strides), same swizzle, rows past the class's extent
+//              zero-filled by TMA.
 //   Both use the same flat row pitch Wzq, which is what makes a tap a pure shift.
-// One thread issues the TMA copies, one thread issues tcgen05.mma, four warps
-// drain the accumulators from tensor memory at the end. K is split over CTAs.
+// Warp 0 issues the TMA copies (one chunk per lane), warps 1 and 6 issue tcgen05.mma (each
+// every second accumulator tile, one elected lane), warps 2-5 drain the accumulators from
+// tensor memory. Every CTA keeps all the accumulator tiles that fit its 512 TMEM columns; K
+// is split over CTAs and the partial dW tensors are summed in a fixed order afterwards.
 #include <cuda.h>
 
 #include <cstring>
@@ -974,17 +981,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
+// Looked up once; the initialisation of a function-local static is thread-safe.
 EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    static const EncodeTiledFn fn = [] {
         void* f = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(f);
-    }
+            return reinterpret_cast<EncodeTiledFn>(f);
+        return static_cast<EncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
 
