@@ -45,6 +45,7 @@ def _load():
         _lib = ctypes.CDLL(_LIB)
         _lib.oracle_num_threads.restype = ctypes.c_int
         _lib.oracle_wgrad_compressed.restype = ctypes.c_int
+        _lib.oracle_wgrad_compressed_rect.restype = ctypes.c_int
     return _lib
 
 
@@ -68,9 +69,15 @@ def out_hw(H, W, R, S, stride, pad):
     return (H + 2 * ph - R) // sh + 1, (W + 2 * pw - S) // sw + 1
 
 
+def _khw(k):
+    """k as (k_h, k_w); an int means a square block."""
+    return (int(k), int(k)) if np.isscalar(k) else (int(k[0]), int(k[1]))
+
+
 def pooled_hw(H, W, k):
-    """Size of Z: partial edge blocks are kept (ceil)."""
-    return -(-H // k), -(-W // k)
+    """Size of Z: partial edge blocks are kept (ceil). k: int, or (k_h, k_w)."""
+    kh, kw = _khw(k)
+    return -(-H // kh), -(-W // kw)
 
 
 def pool(x: np.ndarray, k: int) -> np.ndarray:
@@ -79,6 +86,9 @@ def pool(x: np.ndarray, k: int) -> np.ndarray:
     N, C, H, W = x.shape
     Hp, Wp = pooled_hw(H, W, k)
     z = np.empty((N, C, Hp, Wp), dtype=np.float64)
+    if not np.isscalar(k):      # non-uniform block (k_h, k_w)
+        _load().oracle_pool_rect(_p(x), _i64(N), _i64(C), _i64(H), _i64(W), _i64(k[0]), _i64(k[1]), _p(z))
+        return z
     _load().oracle_pool(_p(x), _i64(N), _i64(C), _i64(H), _i64(W), _i64(k), _p(z))
     return z
 
@@ -89,6 +99,9 @@ def inflate(z: np.ndarray, H: int, W: int, k: int) -> np.ndarray:
     N, C, Hp, Wp = z.shape
     assert (Hp, Wp) == pooled_hw(H, W, k)
     xt = np.empty((N, C, H, W), dtype=np.float64)
+    if not np.isscalar(k):
+        _load().oracle_inflate_rect(_p(z), _i64(N), _i64(C), _i64(H), _i64(W), _i64(k[0]), _i64(k[1]), _p(xt))
+        return xt
     _load().oracle_inflate(_p(z), _i64(N), _i64(C), _i64(H), _i64(W), _i64(k), _p(xt))
     return xt
 
@@ -122,6 +135,14 @@ def wgrad_compressed(z, dy, H, W, R, S, stride=(1, 1), pad=(0, 0), k=2) -> np.nd
     assert z.shape[2:] == pooled_hw(H, W, k)
     assert dy.shape == (N, Co) + out_hw(H, W, R, S, stride, pad)
     dw = np.empty((Co, Ci, R, S), dtype=np.float64)
+    if not np.isscalar(k):
+        rc = _load().oracle_wgrad_compressed_rect(
+            _p(z), _p(dy), _i64(N), _i64(Ci), _i64(Co), _i64(H), _i64(W), _i64(R),
+            _i64(S), _i64(stride[0]), _i64(stride[1]), _i64(pad[0]), _i64(pad[1]),
+            _i64(k[0]), _i64(k[1]), _p(dw))
+        if rc != 0:
+            raise MemoryError("oracle_wgrad_compressed_rect: temporary allocation failed")
+        return dw
     rc = _load().oracle_wgrad_compressed(
         _p(z), _p(dy), _i64(N), _i64(Ci), _i64(Co), _i64(H), _i64(W), _i64(R),
         _i64(S), _i64(stride[0]), _i64(stride[1]), _i64(pad[0]), _i64(pad[1]),
@@ -140,6 +161,12 @@ def wgrad_compressed_entries(z, dy, H, W, R, S, stride, pad, k, idx) -> np.ndarr
     assert z.shape[2:] == pooled_hw(H, W, k)
     assert dy.shape == (N, Co) + out_hw(H, W, R, S, stride, pad)
     out = np.empty(idx.shape[0], dtype=np.float64)
+    if not np.isscalar(k):
+        _load().oracle_wgrad_compressed_rect_entries(
+            _p(z), _p(dy), _i64(N), _i64(Ci), _i64(Co), _i64(H), _i64(W), _i64(R),
+            _i64(S), _i64(stride[0]), _i64(stride[1]), _i64(pad[0]), _i64(pad[1]),
+            _i64(k[0]), _i64(k[1]), idx.ctypes.data_as(_ip), _i64(idx.shape[0]), _p(out))
+        return out
     _load().oracle_wgrad_compressed_entries(
         _p(z), _p(dy), _i64(N), _i64(Ci), _i64(Co), _i64(H), _i64(W), _i64(R),
         _i64(S), _i64(stride[0]), _i64(stride[1]), _i64(pad[0]), _i64(pad[1]),

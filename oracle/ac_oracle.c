@@ -180,6 +180,100 @@ void oracle_wgrad_compressed_entries(const double *z, const double *dy,
     }
 }
 
+/* ---- Non-uniform pooling shapes (Section 6 names them as future work; the
+ * definitions of Section 4 carry over with a k_h x k_w block in place of the
+ * k x k one). Written out separately so that the square functions above stay
+ * exactly as they are. ------------------------------------------------------ */
+
+/* Z[n,c,p,q] = mean of X over rows [p*kh, min((p+1)*kh, H)) and columns
+ * [q*kw, min((q+1)*kw, W)). */
+void oracle_pool_rect(const double *x, int64_t N, int64_t C, int64_t H, int64_t W,
+                      int64_t kh, int64_t kw, double *z)
+{
+    const int64_t Hp = ceil_div(H, kh), Wp = ceil_div(W, kw);
+    #pragma omp parallel for schedule(static)
+    for (int64_t nc = 0; nc < N * C; ++nc) {
+        const double *xp = x + nc * H * W;
+        double *zp = z + nc * Hp * Wp;
+        for (int64_t p = 0; p < Hp; ++p) {
+            for (int64_t q = 0; q < Wp; ++q) {
+                double sum = 0.0;
+                int64_t count = 0;
+                for (int64_t h = p * kh; h < (p + 1) * kh && h < H; ++h) {
+                    for (int64_t w = q * kw; w < (q + 1) * kw && w < W; ++w) {
+                        sum += xp[h * W + w];
+                        ++count;
+                    }
+                }
+                zp[p * Wp + q] = sum / (double)count;
+            }
+        }
+    }
+}
+
+/* Xt[n,c,h,w] = Z[n,c,h/kh,w/kw]. */
+void oracle_inflate_rect(const double *z, int64_t N, int64_t C, int64_t H, int64_t W,
+                         int64_t kh, int64_t kw, double *xt)
+{
+    const int64_t Hp = ceil_div(H, kh), Wp = ceil_div(W, kw);
+    #pragma omp parallel for schedule(static)
+    for (int64_t nc = 0; nc < N * C; ++nc) {
+        const double *zp = z + nc * Hp * Wp;
+        double *xp = xt + nc * H * W;
+        for (int64_t h = 0; h < H; ++h)
+            for (int64_t w = 0; w < W; ++w)
+                xp[h * W + w] = zp[(h / kh) * Wp + (w / kw)];
+    }
+}
+
+/* Inflate by (kh, kw), then the ordinary weight gradient. */
+int oracle_wgrad_compressed_rect(const double *z, const double *dy,
+                                 int64_t N, int64_t Ci, int64_t Co, int64_t H, int64_t W,
+                                 int64_t R, int64_t S, int64_t sh, int64_t sw,
+                                 int64_t ph, int64_t pw, int64_t kh, int64_t kw, double *dw)
+{
+    double *xt = (double *)malloc(sizeof(double) * (size_t)(N * Ci * H * W));
+    if (!xt) return -1;
+    oracle_inflate_rect(z, N, Ci, H, W, kh, kw, xt);
+    oracle_wgrad_dense(xt, dy, N, Ci, Co, H, W, R, S, sh, sw, ph, pw, dw);
+    free(xt);
+    return 0;
+}
+
+/* The same sum at chosen entries idx[4*i..] = (co, ci, r, s), the inflated
+ * value read through the index map h/kh, w/kw. */
+void oracle_wgrad_compressed_rect_entries(const double *z, const double *dy,
+                            int64_t N, int64_t Ci, int64_t Co, int64_t H, int64_t W,
+                            int64_t R, int64_t S, int64_t sh, int64_t sw,
+                            int64_t ph, int64_t pw, int64_t kh, int64_t kw,
+                            const int64_t *idx, int64_t count, double *out)
+{
+    const int64_t Hp = ceil_div(H, kh), Wp = ceil_div(W, kw);
+    const int64_t Ho = (H + 2 * ph - R) / sh + 1;
+    const int64_t Wo = (W + 2 * pw - S) / sw + 1;
+    (void)R; (void)S;
+    #pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < count; ++i) {
+        const int64_t co = idx[4 * i], ci = idx[4 * i + 1];
+        const int64_t r = idx[4 * i + 2], s = idx[4 * i + 3];
+        double acc = 0.0;
+        for (int64_t n = 0; n < N; ++n) {
+            const double *zp = z + (n * Ci + ci) * Hp * Wp;
+            const double *gp = dy + (n * Co + co) * Ho * Wo;
+            for (int64_t ho = 0; ho < Ho; ++ho) {
+                const int64_t h = ho * sh - ph + r;
+                if (h < 0 || h >= H) continue;
+                for (int64_t wo = 0; wo < Wo; ++wo) {
+                    const int64_t w = wo * sw - pw + s;
+                    if (w < 0 || w >= W) continue;
+                    acc += gp[ho * Wo + wo] * zp[(h / kh) * Wp + (w / kw)];
+                }
+            }
+        }
+        out[i] = acc;
+    }
+}
+
 /* Number of OpenMP threads the loops above will use (for reporting). */
 #ifdef _OPENMP
 #include <omp.h>
