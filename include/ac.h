@@ -270,6 +270,30 @@ ac_status ac_conv2d_wgrad_compressed_static(const ac_conv_desc *desc, const void
                                             const void *dy, float *dw, void *stream);
 
 /*
+ * Non-uniform pooling blocks: k_h rows by k_w columns instead of k x k. The
+ * paper (Section 6) lists such shapes as future work; Section 4's definitions
+ * carry over unchanged with Z[n,c,p,q] = mean of X over h in [p k_h,
+ * min((p+1) k_h, H)), w in [q k_w, min((q+1) k_w, W)), Z of size ceil(H/k_h) x
+ * ceil(W/k_w), and Xt[n,c,h,w] = Z[n,c,h/k_h,w/k_w]. The three calls below are
+ * ac_workspace_bytes, ac_compress and ac_conv2d_wgrad_compressed with the block
+ * given beside the descriptor (k_h, k_w >= 1; desc->k is ignored); every other
+ * argument, the layouts, the return codes and the status block are theirs.
+ * k_h == k_w gives bit for bit what the square calls give. With k_h != k_w:
+ * compression runs on the NHWC vector kernel (C_in a multiple of the 16-byte
+ * vector) or the generic kernel; the weight gradient runs on the TMA-fed
+ * tensor-core kernel when stride_h divides k_h and stride_w divides k_w
+ * (bf16 NHWC directly, fp32 / NCHW staged through the workspace), else on the
+ * fp32-ALU kernel. Passing k_h = k_w = 0 means desc->k.
+ */
+size_t ac_workspace_bytes_rect(const ac_conv_desc *desc, int32_t k_h, int32_t k_w);
+ac_status ac_compress_rect(const ac_conv_desc *desc, int32_t k_h, int32_t k_w,
+                           const void *x, void *z, void *y_out, void *stream);
+ac_status ac_conv2d_wgrad_compressed_rect(const ac_conv_desc *desc, int32_t k_h, int32_t k_w,
+                                          const void *z, const void *dy, float *dw,
+                                          void *workspace, size_t workspace_bytes,
+                                          void *stream);
+
+/*
  * How ac_conv2d_wgrad_compressed will run this problem (pure host code; for
  * reports and tests). Returns AC_ERR_INVALID_ARG for an invalid descriptor.
  */

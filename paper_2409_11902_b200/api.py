@@ -92,6 +92,13 @@ def lib() -> ctypes.CDLL:
         L.ac_collapsed_workspace_bytes.argtypes = [dp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
         L.ac_conv2d_wgrad_compressed_collapsed.restype = ctypes.c_int
         L.ac_conv2d_wgrad_compressed_collapsed.argtypes = [dp, vp, vp, vp, vp, sz, vp]
+        i32 = ctypes.c_int32
+        L.ac_workspace_bytes_rect.restype = sz
+        L.ac_workspace_bytes_rect.argtypes = [dp, i32, i32]
+        L.ac_compress_rect.restype = ctypes.c_int
+        L.ac_compress_rect.argtypes = [dp, i32, i32, vp, vp, vp, vp]
+        L.ac_conv2d_wgrad_compressed_rect.restype = ctypes.c_int
+        L.ac_conv2d_wgrad_compressed_rect.argtypes = [dp, i32, i32, vp, vp, vp, vp, sz, vp]
         L.ac_status_string.restype = ctypes.c_char_p
         L.ac_status_string.argtypes = [ctypes.c_int]
         _lib = L
@@ -262,6 +269,29 @@ def ac_conv2d_wgrad_compressed_static(desc: ConvDesc, z, dy, dw, stream=None) ->
                                                  _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_conv2d_wgrad_compressed_static")
+
+
+def ac_workspace_bytes_rect(desc: ConvDesc, k_h: int, k_w: int) -> int:
+    c = desc.c()
+    return int(lib().ac_workspace_bytes_rect(ctypes.byref(c), k_h, k_w))
+
+
+def ac_compress_rect(desc: ConvDesc, k_h: int, k_w: int, x, z, y_out=None, stream=None) -> None:
+    c = desc.c()
+    st = lib().ac_compress_rect(ctypes.byref(c), k_h, k_w, _ptr(x), _ptr(z), _ptr(y_out), _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_compress_rect")
+
+
+def ac_conv2d_wgrad_compressed_rect(desc: ConvDesc, k_h: int, k_w: int, z, dy, dw, workspace,
+                                    workspace_bytes=None, stream=None) -> None:
+    c = desc.c()
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    st = lib().ac_conv2d_wgrad_compressed_rect(ctypes.byref(c), k_h, k_w, _ptr(z), _ptr(dy), _ptr(dw),
+                                               _ptr(workspace), workspace_bytes, _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_conv2d_wgrad_compressed_rect")
 
 
 def ac_wgrad_plan_info(desc: ConvDesc) -> dict:

@@ -57,7 +57,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
         list(pool.map(compile_one, todo))
-    subprocess.run([nvcc, "-shared", "-o", LIB] + [_obj(s) for s in srcs] + ["-lcuda"], check=True)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB]
+                   + [_obj(s) for s in srcs] + ["-lcuda"], check=True)
     return LIB
 
 

@@ -3,17 +3,20 @@
 
 namespace ac {
 
-ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o) {
+ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o, int k_h, int k_w) {
     if (!d || !o) return AC_ERR_INVALID_ARG;
     *o = Dims{};   // plans are cached by the bytes of this struct
-    if (d->N <= 0 || d->C_in <= 0 || d->H <= 0 || d->W <= 0 || d->k <= 0) return AC_ERR_INVALID_ARG;
+    const bool rect = k_h != 0 || k_w != 0;
+    if (rect && (k_h <= 0 || k_w <= 0)) return AC_ERR_INVALID_ARG;
+    if (d->N <= 0 || d->C_in <= 0 || d->H <= 0 || d->W <= 0 || (!rect && d->k <= 0)) return AC_ERR_INVALID_ARG;
     if (d->dtype != AC_F32 && d->dtype != AC_BF16) return AC_ERR_INVALID_ARG;
     if (d->layout != AC_NCHW && d->layout != AC_NHWC) return AC_ERR_INVALID_ARG;
-    o->N = d->N; o->Ci = d->C_in; o->H = d->H; o->W = d->W; o->k = d->k;
+    o->N = d->N; o->Ci = d->C_in; o->H = d->H; o->W = d->W;
+    o->kh = rect ? k_h : d->k; o->kw = rect ? k_w : d->k; o->k = o->kh;
     o->dtype = d->dtype; o->layout = d->layout;
     o->elt = d->dtype == AC_F32 ? 4 : 2;
-    o->Hp = (d->H + d->k - 1) / d->k;
-    o->Wp = (d->W + d->k - 1) / d->k;
+    o->Hp = (d->H + o->kh - 1) / o->kh;
+    o->Wp = (d->W + o->kw - 1) / o->kw;
     o->Co = 1; o->R = 1; o->S = 1; o->sh = 1; o->sw = 1; o->ph = 0; o->pw = 0;
     o->Ho = d->H; o->Wo = d->W;
     const long long lim = 1ll << 40;  // elements; far above 180 GB of any dtype
@@ -114,9 +117,11 @@ using namespace ac;
 
 extern "C" {
 
-size_t ac_workspace_bytes(const ac_conv_desc* desc) {
+size_t ac_workspace_bytes(const ac_conv_desc* desc) { return ac_workspace_bytes_rect(desc, 0, 0); }
+
+size_t ac_workspace_bytes_rect(const ac_conv_desc* desc, int32_t k_h, int32_t k_w) {
     Dims d;
-    if (make_dims(desc, true, &d) != AC_OK) return 0;
+    if (make_dims(desc, true, &d, k_h, k_w) != AC_OK) return 0;
     return plan_wgrad(d).bytes;
 }
 
@@ -128,8 +133,13 @@ size_t ac_workspace_bytes_min(const ac_conv_desc* desc) {
 }
 
 ac_status ac_compress(const ac_conv_desc* desc, const void* x, void* z, void* y_out, void* stream) {
+    return ac_compress_rect(desc, 0, 0, x, z, y_out, stream);
+}
+
+ac_status ac_compress_rect(const ac_conv_desc* desc, int32_t k_h, int32_t k_w, const void* x, void* z,
+                           void* y_out, void* stream) {
     Dims d;
-    ac_status st = make_dims(desc, false, &d);
+    ac_status st = make_dims(desc, false, &d, k_h, k_w);
     if (st != AC_OK) return st;
     if (!x || !z) return AC_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(z) || !aligned16(y_out)) return AC_ERR_MISALIGNED;
@@ -149,8 +159,14 @@ ac_status ac_compress_relu_mask(const ac_conv_desc* desc, const void* a, void* z
 ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, const void* dy,
                                      float* dw, void* workspace, size_t workspace_bytes,
                                      void* stream) {
+    return ac_conv2d_wgrad_compressed_rect(desc, 0, 0, z, dy, dw, workspace, workspace_bytes, stream);
+}
+
+ac_status ac_conv2d_wgrad_compressed_rect(const ac_conv_desc* desc, int32_t k_h, int32_t k_w, const void* z,
+                                          const void* dy, float* dw, void* workspace,
+                                          size_t workspace_bytes, void* stream) {
     Dims d;
-    ac_status st = make_dims(desc, true, &d);
+    ac_status st = make_dims(desc, true, &d, k_h, k_w);
     if (st != AC_OK) return st;
     if (!z || !dy || !dw || !workspace) return AC_ERR_INVALID_ARG;
     if (!aligned16(z) || !aligned16(dy) || !aligned16(dw) || !aligned16(workspace))

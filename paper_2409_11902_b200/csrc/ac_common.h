@@ -15,6 +15,8 @@ constexpr size_t kStatusBlockBytes = 256;  // first bytes of every wgrad workspa
 // Derived sizes of a validated descriptor.
 struct Dims {
     int N, Ci, Co, H, W, R, S, sh, sw, ph, pw, k;
+    int kh, kw;   // pooling block; k = kh = kw for the square blocks of the paper. Code that reads
+                  // only `k` must not be reached with kh != kw (each path's *_supported says so).
     int Hp, Wp;   // pooled size (ceil)
     int Ho, Wo;   // convolution output size
     int dtype, layout;
@@ -33,7 +35,8 @@ struct Dims {
 
 // Validates and expands a descriptor. `need_conv` = false checks only the
 // fields ac_compress uses.
-ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* out);
+// k_h, k_w > 0: a non-uniform pooling block, desc->k is then ignored.
+ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* out, int k_h = 0, int k_w = 0);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -130,7 +130,7 @@ __device__ __forceinline__ void store_mask(unsigned char* mask, long long elem_o
 template <typename T, int K, int MODE>   // MODE 0: pool only, 1: also store max(x,0), 2: also store the sign mask
 __global__ void __launch_bounds__(256)
 compress_nhwc_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int CV,
-                  int k, int Hp, int Wp) {
+                  int kh, int kw, int Hp, int Wp) {
     pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
     constexpr bool RELU = MODE != 0;
     constexpr int VW = VecTraits<T>::VW;
@@ -142,9 +142,9 @@ compress_nhwc_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int 
     const int cv = (int)(item - (unsigned)q * (unsigned)CV);
     const int p = blockIdx.y;
     const long long n = blockIdx.z;
-    const int kk = K > 0 ? K : k;
-    const int h0 = p * kk, w0 = q * kk;
-    const int h1 = min(h0 + kk, H), w1 = min(w0 + kk, W);
+    const int kkh = K > 0 ? K : kh, kkw = K > 0 ? K : kw;   // K = 0 also serves blocks with kh != kw
+    const int h0 = p * kkh, w0 = q * kkw;
+    const int h1 = min(h0 + kkh, H), w1 = min(w0 + kkw, W);
     float acc[VW];
 #pragma unroll
     for (int i = 0; i < VW; ++i) acc[i] = 0.f;
@@ -211,19 +211,19 @@ compress_nhwc_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int 
 }
 
 template <typename T, int MODE>
-ac_status launch_nhwc_vec(const T* x, T* z, T* y, unsigned char* mask, long long N, int H, int W, int CV, int k,
-                          int Hp, int Wp, cudaStream_t st) {
+ac_status launch_nhwc_vec(const T* x, T* z, T* y, unsigned char* mask, long long N, int H, int W, int CV, int kh,
+                          int kw, int Hp, int Wp, cudaStream_t st) {
     const long long row_items = (long long)Wp * CV;
     if (row_items >= (1ll << 31) || Hp > 65535 || N > 65535) return AC_ERR_UNSUPPORTED;
     dim3 grid((unsigned)((row_items + 255) / 256), (unsigned)Hp, (unsigned)N);
-    switch (k) {
-        case 1: compress_nhwc_vec<T, 1, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp); break;
-        case 2: compress_nhwc_vec<T, 2, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp); break;
-        case 4: compress_nhwc_vec<T, 4, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp); break;
-        case 8: compress_nhwc_vec<T, 8, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp); break;
+    switch (kh == kw ? kh : 0) {
+        case 1: compress_nhwc_vec<T, 1, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, kh, kw, Hp, Wp); break;
+        case 2: compress_nhwc_vec<T, 2, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, kh, kw, Hp, Wp); break;
+        case 4: compress_nhwc_vec<T, 4, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, kh, kw, Hp, Wp); break;
+        case 8: compress_nhwc_vec<T, 8, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, kh, kw, Hp, Wp); break;
         default:
             if (MODE == 2) return AC_ERR_UNSUPPORTED;   // the mask needs warp-uniform loops
-            compress_nhwc_vec<T, 0, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, k, Hp, Wp);
+            compress_nhwc_vec<T, 0, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, kh, kw, Hp, Wp);
             break;
     }
     AC_CUDA_TRY(cudaGetLastError());
@@ -305,7 +305,7 @@ compress_nchw_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int 
 // ---- any layout, any k, any size: one thread per element of Z ---------------
 template <typename T, bool RELU>
 __global__ void __launch_bounds__(256)
-compress_generic(const T* x, T* __restrict__ z, T* y, int C, int H, int W, int k, int Hp, int Wp,
+compress_generic(const T* x, T* __restrict__ z, T* y, int C, int H, int W, int kh, int kw, int Hp, int Wp,
                  int nhwc, long long total) {
     pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -314,8 +314,8 @@ compress_generic(const T* x, T* __restrict__ z, T* y, int C, int H, int W, int k
     long long n, t = idx;
     if (nhwc) { c = (int)(t % C); t /= C; q = (int)(t % Wp); t /= Wp; p = (int)(t % Hp); n = t / Hp; }
     else      { q = (int)(t % Wp); t /= Wp; p = (int)(t % Hp); t /= Hp; c = (int)(t % C); n = t / C; }
-    const int h0 = p * k, w0 = q * k;
-    const int h1 = min(h0 + k, H), w1 = min(w0 + k, W);
+    const int h0 = p * kh, w0 = q * kw;
+    const int h1 = min(h0 + kh, H), w1 = min(w0 + kw, W);
     float acc = 0.f;
     for (int h = h0; h < h1; ++h) {
         float row = 0.f;
@@ -351,16 +351,17 @@ ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, unsigned char* mas
     constexpr int VW = VecTraits<T>::VW;
     const long long zt = d.z_elems();
     if (zt >= (1ll << 31) * 256) return AC_ERR_UNSUPPORTED;
-    const bool pow2k = d.k == 2 || d.k == 4 || d.k == 8;
-    if (d.k == 1 && d.x_elems() % (MODE == 2 ? 8 : VW) == 0) {
+    const bool square = d.kh == d.kw;
+    const bool pow2k = square && (d.k == 2 || d.k == 4 || d.k == 8);
+    if (square && d.k == 1 && d.x_elems() % (MODE == 2 ? 8 : VW) == 0) {
         // a copy (or a plain ReLU): treat the tensor as one row of 16-byte vectors
         const long long nv = d.x_elems() / VW;
         if (nv < (1ll << 31))
-            return launch_nhwc_vec<T, MODE>(x, z, y, mask, 1, 1, (int)nv, 1, 1, 1, (int)nv, st);
+            return launch_nhwc_vec<T, MODE>(x, z, y, mask, 1, 1, (int)nv, 1, 1, 1, 1, (int)nv, st);
     }
     if (d.layout == AC_NHWC && d.Ci % (MODE == 2 ? 8 : VW) == 0) {
         const ac_status st_ =
-            launch_nhwc_vec<T, MODE>(x, z, y, mask, d.N, d.H, d.W, d.Ci / VW, d.k, d.Hp, d.Wp, st);
+            launch_nhwc_vec<T, MODE>(x, z, y, mask, d.N, d.H, d.W, d.Ci / VW, d.kh, d.kw, d.Hp, d.Wp, st);
         if (st_ != AC_ERR_UNSUPPORTED) return st_;
     }
     if (d.layout == AC_NCHW && pow2k && d.W % (MODE == 2 ? 8 : VW) == 0 && d.W % d.k == 0 &&
@@ -372,7 +373,7 @@ ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, unsigned char* mas
     } else {
         if (MODE == 2) return AC_ERR_UNSUPPORTED;
         compress_generic<T, MODE != 0><<<blocks_for(zt), 256, 0, st>>>(
-            x, z, y, d.Ci, d.H, d.W, d.k, d.Hp, d.Wp, d.layout == AC_NHWC, zt);
+            x, z, y, d.Ci, d.H, d.W, d.kh, d.kw, d.Hp, d.Wp, d.layout == AC_NHWC, zt);
     }
     AC_CUDA_TRY(cudaGetLastError());
     return AC_OK;

@@ -27,7 +27,7 @@ __device__ __forceinline__ float ldf(const __nv_bfloat16* p, long long i) {
 }
 
 struct SimtParams {
-    int N, Ci, Co, H, W, R, S, sh, sw, ph, pw, k, Hp, Wp, Ho, Wo;
+    int N, Ci, Co, H, W, R, S, sh, sw, ph, pw, kh, kw, Hp, Wp, Ho, Wo;
     int nhwc;
     int J;                 // Ci*R*S
     long long K;           // N*Ho*Wo
@@ -94,7 +94,7 @@ wgrad_simt_kernel(const T* __restrict__ z, const T* __restrict__ dy, float* __re
                 const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
                 const int h = ho * p.sh - p.ph + r, w = wo * p.sw - p.pw + s;
                 if (h >= 0 && h < p.H && w >= 0 && w < p.W) {
-                    const int hp = h / p.k, wp = w / p.k;
+                    const int hp = h / p.kh, wp = w / p.kw;
                     const long long off =
                         p.nhwc ? ((n * p.Hp + hp) * (long long)p.Wp + wp) * p.Ci + ci
                                : ((n * p.Ci + ci) * (long long)p.Hp + hp) * p.Wp + wp;
@@ -252,7 +252,7 @@ ac_status launch_wgrad_simt(const Dims& d, const WgradPlan& pl, const void* z, c
                             float* dw, void* workspace, cudaStream_t stream) {
     SimtParams p;
     p.N = d.N; p.Ci = d.Ci; p.Co = d.Co; p.H = d.H; p.W = d.W; p.R = d.R; p.S = d.S;
-    p.sh = d.sh; p.sw = d.sw; p.ph = d.ph; p.pw = d.pw; p.k = d.k; p.Hp = d.Hp; p.Wp = d.Wp;
+    p.sh = d.sh; p.sw = d.sw; p.ph = d.ph; p.pw = d.pw; p.kh = d.kh; p.kw = d.kw; p.Hp = d.Hp; p.Wp = d.Wp;
     p.Ho = d.Ho; p.Wo = d.Wo; p.nhwc = d.layout == AC_NHWC;
     p.J = d.Ci * d.R * d.S;
     p.K = d.K();

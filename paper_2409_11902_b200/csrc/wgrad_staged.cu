@@ -358,6 +358,7 @@ GatherGeom gather_geom(const Dims& d) {
     if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
     if (d.Ci >= 64 || d.Co % 64 != 0) return g;
     if (d.R > 255 || d.S > 255) return g;
+    if (d.kh != d.kw) return g;      // the gather's index map knows square pooling blocks only
     GatherParams& p = g.p;
     p.Ci = d.Ci; p.H = d.H; p.W = d.W; p.Hp = d.Hp; p.Wp = d.Wp; p.Ho = d.Ho; p.Wo = d.Wo; p.k = d.k;
     p.sh = d.sh; p.sw = d.sw; p.ph = d.ph; p.pw = d.pw;
@@ -390,7 +391,7 @@ GatherGeom gather_geom(const Dims& d) {
     in.R = in.S = 1;
     in.sh = in.sw = 1;
     in.ph = in.pw = 0;
-    in.k = 1;
+    in.k = in.kh = in.kw = 1;
     g.in = in;
     g.ok = tc2_supported(in, nullptr);
     return g;

@@ -294,6 +294,7 @@ TcGeom make_geom(const Dims& d) {
     g.ok = false;
     if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
     if (d.Ci % 64 != 0 || d.Co % 64 != 0) return g;
+    if (d.kh != d.kw) return g;      // the producer warps' index map knows square pooling blocks only
     if (d.sh < 1 || d.sh > 2 || d.sw < 1 || d.sw > 2) return g;
     if (d.R * d.S > 64) return g;
     p.N = d.N; p.Ci = d.Ci; p.Co = d.Co; p.H = d.H; p.W = d.W; p.R = d.R; p.S = d.S;

@@ -63,7 +63,7 @@ struct Tc2Params {
     float* out;
     uint32_t* status;
     int keep_status;   // 1: a launch earlier in the same call owns the status block; do not reset it
-    int Ci, Co, R, S, sh, sw, ph, pw, k;
+    int Ci, Co, R, S, sh, sw, ph, pw, kh, kw;   // pooling block kh x kw (square in the paper: kh = kw = k)
     int c_h, c_w, ncls;
     int umin, vmin;
     int Wzq, Ic, bands, KT, ksteps, rowsA;
@@ -121,13 +121,13 @@ __host__ __device__ inline bool reads_padding_in_partial_block(int s, int a, int
 // (u = floor((s_h*a - p_h + r) / k) is non-decreasing in r with steps of 0 or 1).
 struct ClassShifts { int u0, nU, v0, nV; };
 __host__ __device__ inline ClassShifts class_shifts(int cls, int c_w, int sh, int sw, int ph, int pw,
-                                                    int k, int R, int S) {
+                                                    int kh, int kw, int R, int S) {
     const int a = cls / c_w, b = cls - a * c_w;
     ClassShifts c;
-    c.u0 = floor_div_i(sh * a - ph, k);
-    c.nU = floor_div_i(sh * a - ph + R - 1, k) - c.u0 + 1;
-    c.v0 = floor_div_i(sw * b - pw, k);
-    c.nV = floor_div_i(sw * b - pw + S - 1, k) - c.v0 + 1;
+    c.u0 = floor_div_i(sh * a - ph, kh);
+    c.nU = floor_div_i(sh * a - ph + R - 1, kh) - c.u0 + 1;
+    c.v0 = floor_div_i(sw * b - pw, kw);
+    c.nV = floor_div_i(sw * b - pw + S - 1, kw) - c.v0 + 1;
     return c;
 }
 
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         int base = 0;
         cls0 = -1;
         for (int c = 0; c < p.ncls; ++c) {
-            const ClassShifts cs = class_shifts(c, p.c_w, p.sh, p.sw, p.ph, p.pw, p.k, p.R, p.S);
+            const ClassShifts cs = class_shifts(c, p.c_w, p.sh, p.sw, p.ph, p.pw, p.kh, p.kw, p.R, p.S);
             const int cnt = cs.nU * cs.nV;
             if (cls0 < 0 && base + cnt > cj0) cls0 = c;
             if (base < cj0 + cn) cls1 = c + 1;
@@ -333,7 +333,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             // tile u = number cj0 + u: find its class and its shift inside the class
             int base = 0, u = 0;
             for (int c = 0; c < p.ncls && u < nunits; ++c) {
-                const ClassShifts cs = class_shifts(c, p.c_w, p.sh, p.sw, p.ph, p.pw, p.k, p.R, p.S);
+                const ClassShifts cs = class_shifts(c, p.c_w, p.sh, p.sw, p.ph, p.pw, p.kh, p.kw, p.R, p.S);
                 const int cnt = cs.nU * cs.nV;
                 while (u < nunits && cj0 + u < base + cnt) {
                     const int j = cj0 + u - base, iu = j / cs.nV, iv = j - iu * cs.nV;
@@ -353,12 +353,12 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 const int cl = u / ntap, t = u - cl * ntap;
                 const int tap = tap0 + t, r = tap / p.S, sx = tap - r * p.S;
                 const int a = cls / p.c_w, b = cls - a * p.c_w;
-                const int uu = floor_div_i(p.sh * a - p.ph + r, p.k) - p.umin;
-                const int vv = floor_div_i(p.sw * b - p.pw + sx, p.k) - p.vmin;
+                const int uu = floor_div_i(p.sh * a - p.ph + r, p.kh) - p.umin;
+                const int vv = floor_div_i(p.sw * b - p.pw + sx, p.kw) - p.vmin;
                 // which copy of the tile: the one without the partial last row / column of Z if this
                 // (class, tap) reaches past H / W there
-                const int var = (reads_padding_in_partial_block(p.sh, a, p.ph, r, p.k, p.Hp, p.rho_h, p.Ho) ? 2 : 0) +
-                                (reads_padding_in_partial_block(p.sw, b, p.pw, sx, p.k, p.Wp, p.rho_w, p.Wo) ? 1 : 0);
+                const int var = (reads_padding_in_partial_block(p.sh, a, p.ph, r, p.kh, p.Hp, p.rho_h, p.Ho) ? 2 : 0) +
+                                (reads_padding_in_partial_block(p.sw, b, p.pw, sx, p.kw, p.Wp, p.rho_w, p.Wo) ? 1 : 0);
                 off = (uint32_t)(p.var_slot[var] * p.chunksA + cl * (p.CB / 64)) * p.a_chunk_bytes +
                       (uint32_t)(uu * p.Wzq + vv) * 128u;
             }
@@ -526,7 +526,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
 //   that class. One float4 of ci per thread group; SL threads share the (class, slice) pairs,
 // each adding its pairs in order, then the SL running sums are added in index order.
 struct CollapseReduceParams {
-    int splits, ncls, R, S, Ci, CB, BN, ncib_total, cu_total, c_w, sh, sw, ph, pw, k;
+    int splits, ncls, R, S, Ci, CB, BN, ncib_total, cu_total, c_w, sh, sw, ph, pw, kh, kw;
     long long slice_elems, elems4;
 };
 
@@ -543,13 +543,13 @@ collapsed_reduce_kernel(const float4* __restrict__ P, CollapseReduceParams q, fl
             const int cls = e / RS, tap = e - cls * RS, r = tap / q.S, sx = tap - r * q.S;
             int base = 0;
             for (int c = 0; c < cls; ++c) {
-                const ClassShifts cs = class_shifts(c, q.c_w, q.sh, q.sw, q.ph, q.pw, q.k, q.R, q.S);
+                const ClassShifts cs = class_shifts(c, q.c_w, q.sh, q.sw, q.ph, q.pw, q.kh, q.kw, q.R, q.S);
                 base += cs.nU * cs.nV;
             }
-            const ClassShifts cs = class_shifts(cls, q.c_w, q.sh, q.sw, q.ph, q.pw, q.k, q.R, q.S);
+            const ClassShifts cs = class_shifts(cls, q.c_w, q.sh, q.sw, q.ph, q.pw, q.kh, q.kw, q.R, q.S);
             const int a = cls / q.c_w, b = cls - a * q.c_w;
-            const int iu = floor_div_i(q.sh * a - q.ph + r, q.k) - cs.u0;
-            const int iv = floor_div_i(q.sw * b - q.pw + sx, q.k) - cs.v0;
+            const int iu = floor_div_i(q.sh * a - q.ph + r, q.kh) - cs.u0;
+            const int iv = floor_div_i(q.sw * b - q.pw + sx, q.kw) - cs.v0;
             jmap[e] = (unsigned short)(base + iu * cs.nV + iv);
         }
     }
@@ -644,8 +644,8 @@ bool plan_pairs(const Dims& d, int c_h, int c_w, int umin, int vmin, int uspan, 
     for (int c = 0; c < C; ++c)
         for (int t = 0; t < T; ++t) {
             const int a = c / c_w, b = c % c_w, r = t / d.S, sx = t % d.S;
-            ou[c][t] = floor_div_i(d.sh * a - d.ph + r, d.k) - umin;
-            ov[c][t] = floor_div_i(d.sw * b - d.pw + sx, d.k) - vmin;
+            ou[c][t] = floor_div_i(d.sh * a - d.ph + r, d.kh) - umin;
+            ov[c][t] = floor_div_i(d.sw * b - d.pw + sx, d.kw) - vmin;
         }
     auto diff = [&](int t1, int t2, int* du, int* dv) {   // constant over classes?
         *du = ou[0][t2] - ou[0][t1]; *dv = ov[0][t2] - ov[0][t1];
@@ -740,27 +740,27 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     Tc2Params& p = g.p;
     g.ok = false;
     if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
-    if (d.k % d.sh != 0 || d.k % d.sw != 0) return g;      // class rows advance Z by exactly one row
+    if (d.kh % d.sh != 0 || d.kw % d.sw != 0) return g;    // class rows advance Z by exactly one row
     if (d.R * d.S > 64 || d.R > 16 || d.S > 16) return g;
     const UnitPlan up = plan_units(d.Ci, d.Co, d.R * d.S, kMaxUnits2, fill_rectangles, bn_cap);
     if (!up.ok) return g;
-    p.c_h = d.k / d.sh; p.c_w = d.k / d.sw;
+    p.c_h = d.kh / d.sh; p.c_w = d.kw / d.sw;
     p.ncls = p.c_h * p.c_w;
     if (p.ncls > kMaxClasses) return g;
     p.strided_map = p.ncls > kMaxClassMaps ? 1 : 0;
     if (d.Ho < p.c_h || d.Wo < p.c_w) return g;            // every class has at least one output
     p.Ci = d.Ci; p.Co = d.Co; p.R = d.R; p.S = d.S; p.sh = d.sh; p.sw = d.sw; p.ph = d.ph; p.pw = d.pw;
-    p.k = d.k;
+    p.kh = d.kh; p.kw = d.kw;
     p.dw_elems = d.dw_elems();
     int umin = 1 << 30, umax = -(1 << 30), vmin = 1 << 30, vmax = -(1 << 30);
     for (int a = 0; a < p.c_h; ++a)
         for (int r = 0; r < d.R; ++r) {
-            const int u = floor_div_i(d.sh * a - d.ph + r, d.k);
+            const int u = floor_div_i(d.sh * a - d.ph + r, d.kh);
             umin = u < umin ? u : umin; umax = u > umax ? u : umax;
         }
     for (int b = 0; b < p.c_w; ++b)
         for (int s = 0; s < d.S; ++s) {
-            const int v = floor_div_i(d.sw * b - d.pw + s, d.k);
+            const int v = floor_div_i(d.sw * b - d.pw + s, d.kw);
             vmin = v < vmin ? v : vmin; vmax = v > vmax ? v : vmax;
         }
     p.umin = umin; p.vmin = vmin;
@@ -776,15 +776,15 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     p.tmem_cols = up.tmem_cols;
     int chunksA = up.CB == 128 ? 2 * up.cibs_per_group : up.cibs_per_group + 1;
     // which copies of the Z tile are needed (see Tc2Params::nvar)
-    p.rho_h = d.H % d.k; p.rho_w = d.W % d.k;
+    p.rho_h = d.H % d.kh; p.rho_w = d.W % d.kw;
     p.Hp = d.Hp; p.Wp = d.Wp; p.Ho = d.Ho; p.Wo = d.Wo;
     bool var_used[4] = {false, false, false, false};
     for (int a = 0; a < p.c_h; ++a)
         for (int r = 0; r < d.R; ++r)
             for (int b = 0; b < p.c_w; ++b)
                 for (int s_ = 0; s_ < d.S; ++s_) {
-                    var_used[(reads_padding_in_partial_block(d.sh, a, d.ph, r, d.k, d.Hp, p.rho_h, d.Ho) ? 2 : 0) +
-                             (reads_padding_in_partial_block(d.sw, b, d.pw, s_, d.k, d.Wp, p.rho_w, d.Wo) ? 1 : 0)] = true;
+                    var_used[(reads_padding_in_partial_block(d.sh, a, d.ph, r, d.kh, d.Hp, p.rho_h, d.Ho) ? 2 : 0) +
+                             (reads_padding_in_partial_block(d.sw, b, d.pw, s_, d.kw, d.Wp, p.rho_w, d.Wo) ? 1 : 0)] = true;
                 }
     p.nvar = 0;
     for (int v = 0; v < 4; ++v) p.var_slot[v] = var_used[v] ? p.nvar++ : -1;
@@ -819,7 +819,7 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
         if (p.nvar != 1) return g;
         int total = 0;
         for (int c = 0; c < p.ncls; ++c) {
-            const ClassShifts cs = class_shifts(c, p.c_w, d.sh, d.sw, d.ph, d.pw, d.k, d.R, d.S);
+            const ClassShifts cs = class_shifts(c, p.c_w, d.sh, d.sw, d.ph, d.pw, d.kh, d.kw, d.R, d.S);
             total += cs.nU * cs.nV;
         }
         if (total >= p.ncls * d.R * d.S || total > 65535 || p.ncls * d.R * d.S > 8192) return g;
@@ -893,8 +893,8 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
             const int gq = pairs.grp[u], t = pairs.tapA[u], r = t / d.S, sx = t % d.S;
             for (int c = 0; c < p.ncls; ++c) {
                 const int a = c / p.c_w, b = c % p.c_w;
-                const int ouA = floor_div_i(d.sh * a - d.ph + r, d.k) - umin - pairs.cu[gq];
-                const int ovA = floor_div_i(d.sw * b - d.pw + sx, d.k) - vmin - pairs.cv[gq];
+                const int ouA = floor_div_i(d.sh * a - d.ph + r, d.kh) - umin - pairs.cu[gq];
+                const int ovA = floor_div_i(d.sw * b - d.pw + sx, d.kw) - vmin - pairs.cv[gq];
                 p.pu_off[c][u] = (uint32_t)gq * p.a_chunk_bytes + (uint32_t)(ouA * p.Wzq + ovA) * 128u;
             }
         }
@@ -1105,7 +1105,7 @@ static ac_status launch_tc2_any(const Dims& d, bool collapse, const void* z, con
         CollapseReduceParams q;
         q.splits = p.splits; q.ncls = p.ncls; q.R = d.R; q.S = d.S; q.Ci = d.Ci; q.CB = p.CB; q.BN = p.BN;
         q.ncib_total = p.ncib_total; q.cu_total = p.cu_total; q.c_w = p.c_w; q.sh = d.sh; q.sw = d.sw;
-        q.ph = d.ph; q.pw = d.pw; q.k = d.k; q.slice_elems = p.slice_elems; q.elems4 = p.dw_elems / 4;
+        q.ph = d.ph; q.pw = d.pw; q.kh = d.kh; q.kw = d.kw; q.slice_elems = p.slice_elems; q.elems4 = p.dw_elems / 4;
         const int pairs = p.ncls * p.splits;
         int sl = 1;
         while (sl < 32 && q.elems4 * sl < 148 * 1024 && sl * 4 <= pairs) sl *= 2;

@@ -240,3 +240,22 @@ def test_layer_report_tables_match_the_network():
     table_flops = sum(cnt * 2 * ((H + 2 * pd - R) // st + 1) ** 2 * co * ci * R * R
                       for ci, co, H, R, st, pd, cnt in lr.RESNET50)
     assert table_flops == flops
+
+
+def test_rect_entry_points_validate_the_block(ac):
+    """Needs no GPU: sizes and argument checks of the k_h x k_w calls are host code."""
+    L = ac.api.lib()
+    d = ac.ConvDesc(4, 64, 64, 20, 20, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
+    assert ac.ac_workspace_bytes_rect(d, 2, 2) == ac.ac_workspace_bytes(d)
+    assert ac.ac_workspace_bytes_rect(d, 0, 0) == ac.ac_workspace_bytes(d)
+    assert ac.ac_workspace_bytes_rect(d, 2, 4) >= 256
+    for bad in ((0, 2), (2, 0), (-1, 2), (2, -3)):
+        assert ac.ac_workspace_bytes_rect(d, *bad) == 0
+        c = d.c()
+        A = 0x10000
+        assert L.ac_compress_rect(ctypes.byref(c), bad[0], bad[1], A, A, None, None) == ac.api.AC_ERR_INVALID_ARG
+        assert L.ac_conv2d_wgrad_compressed_rect(ctypes.byref(c), bad[0], bad[1], A, A, A, A, 1 << 30, None) \
+            == ac.api.AC_ERR_INVALID_ARG
+    c = d.c()
+    assert L.ac_conv2d_wgrad_compressed_rect(ctypes.byref(c), 2, 4, 0x10000, 0x10000, 0x10000, 0x10000, 16, None) \
+        == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
