@@ -32,6 +32,7 @@
 // is split over CTAs and the partial dW tensors are summed in a fixed order afterwards.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -44,8 +45,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads2 = 224;        // warp 0: TMA, warps 1 and 6: MMA (1 owns TMEM), warps 2-5: epilogue
-constexpr int kMmaWarps = 2;          // each issues the MMAs of every second accumulator tile
+constexpr int kThreads2 = 224;        // warp 0: TMA, warps 1 and 6: MMA (1 owns TMEM), warps 2-5: epilogue (and MMA)
+constexpr int kMaxMmaWarps = 6;       // accumulator tiles are dealt out over up to this many issuing warps
 constexpr int kMaxUnits2 = 8;
 constexpr int kMaxClasses = 64;      // output classes (k/s_h * k/s_w), e.g. k = 8 at stride 1
 constexpr int kMaxClassMaps = 16;    // classes that get a tensor map of their own
@@ -133,6 +134,21 @@ __host__ __device__ inline ClassShifts class_shifts(int cls, int c_w, int sh, in
 
 extern __shared__ __align__(1024) unsigned char tc2_smem[];
 
+// Development aid, compiled in only with -DAC_TC2_TRACE (never in the library as built by
+// build.py): per-CTA clock stamps and wait totals, read back with ac_debug_read_trace.
+#ifdef AC_TC2_TRACE
+constexpr int kTraceWords = 32;
+__device__ long long g_trace[kNumSMs * 2 * kTraceWords];
+#define TRACE_SET(slot, value) do { if (blockIdx.x < kNumSMs * 2) g_trace[blockIdx.x * kTraceWords + (slot)] = (value); } while (0)
+#define TRACE_ADD(slot, value) do { if (blockIdx.x < kNumSMs * 2) g_trace[blockIdx.x * kTraceWords + (slot)] += (value); } while (0)
+#define TRACE_CLOCK() clock64()
+__device__ __forceinline__ long long trace_gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#else
+#define TRACE_SET(slot, value) do { } while (0)
+#define TRACE_ADD(slot, value) do { } while (0)
+#define TRACE_CLOCK() 0ll
+#endif
+
 __device__ __forceinline__ void flag_timeout(int* abort_s, uint32_t* status, uint32_t code) {
     if (atomicExch(abort_s, 1) == 0) {
         status[1] = code;
@@ -166,6 +182,13 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     volatile int* abort_flag = &abort_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef AC_TC2_TRACE
+    const long long tr_t0 = clock64();
+    if (tid == 0) {
+        for (int i = 0; i < kTraceWords; ++i) TRACE_SET(i, 0);
+        TRACE_SET(0, trace_gtime());
+    }
+#endif
     const int group = blockIdx.x % p.groups, split = blockIdx.x / p.groups;
     const int tg = group % p.ntapgroups;
     const int cibg = (group / p.ntapgroups) % p.ncibgroups;
@@ -197,6 +220,14 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     const int kt_begin = (int)((long long)p.ktiles * split / p.splits);
     const int kt_end = (int)((long long)p.ktiles * (split + 1) / p.splits);
     const int chunk_kt = p.chunk_kt > 0 ? p.chunk_kt : 0x7fffffff;
+    // MMA-issuing warps. An issuing warp that turns to another accumulator tile stalls for a few
+    // hundred cycles (measured: ~280, whatever the tile's width) while MMAs of other warps go on
+    // undisturbed, so every tile gets a warp of its own where possible: warps 1 and 6, then the four
+    // epilogue warps, which have nothing else to do until the accumulators are complete. When the
+    // accumulators are written out in the middle of the K-slice (chunk_kt), the epilogue warps must
+    // stay free for that, and warps 1 and 6 share the tiles.
+    const int nmw = p.chunk_kt > 0 ? 2 : min(max(nunits, 1), kMaxMmaWarps);
+    const int mw = warp == 1 ? 0 : (warp == 6 ? 1 : warp);      // this warp's place among them (warp 0: none)
     // 1024-byte aligned tile area: A slots first, then B slots
     const uint32_t smem_base = (smem_u32(tc2_smem) + 1023u) & ~1023u;
     unsigned char* smem_gen = tc2_smem + (smem_base - smem_u32(tc2_smem));
@@ -221,7 +252,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 const int sa = pr_ta % kSlotsA;
                 if (pr_ta >= kSlotsA) {
                     if (!may_wait) return;
+                    [[maybe_unused]] const long long tw = TRACE_CLOCK();
                     const bool got = mbar_wait(&emptyA[sa], ((pr_ta / kSlotsA) & 1) ^ 1, abort_flag);
+                    if (lane == 0) TRACE_ADD(8, TRACE_CLOCK() - tw);
                     if (!__all_sync(0xffffffffu, got)) {
                         if (lane == 0) flag_timeout(&abort_s, p.status, 0x100u + sa);
                         return;
@@ -245,7 +278,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 const int sb = pr_tb % p.slotsB;
                 if (pr_tb >= p.slotsB) {
                     if (!may_wait) return;
+                    [[maybe_unused]] const long long tw = TRACE_CLOCK();
                     const bool got = mbar_wait(&emptyB[sb], ((pr_tb / p.slotsB) & 1) ^ 1, abort_flag);
+                    if (lane == 0) TRACE_ADD(9, TRACE_CLOCK() - tw);
                     if (!__all_sync(0xffffffffu, got)) {
                         if (lane == 0) flag_timeout(&abort_s, p.status, 0x180u + sb);
                         return;
@@ -283,9 +318,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             prefetch_tmap(&p.tmB[lane - 4]);
         }
         if (lane == 0) {
-            for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], kMmaWarps); }
-            for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], kMmaWarps); }
-            mbar_init(&done_bar, kMmaWarps);
+            for (int s = 0; s < kSlotsA; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], nmw); }
+            for (int s = 0; s < p.slotsB; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], nmw); }
+            mbar_init(&done_bar, nmw);
             mbar_init(&tfree_bar, 4);
             abort_s = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -303,6 +338,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         // can run out (a wait gives up only after 2^32 cycles).
         if (blockIdx.x == 0 && lane == 0 && !p.keep_status) { p.status[0] = 0u; p.status[1] = 0u; }
         produce(true);
+        if (lane == 0) TRACE_SET(10, TRACE_CLOCK() - tr_t0);    // producer done
     }
     // Everything the MMAs may read but no copy ever writes must be finite (it only
     // ever meets zeros of the other operand, or feeds accumulator rows that are
@@ -371,13 +407,12 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         bar_sync(1, kThreads2);
         tc_fence_after();
         tmem_base = tmem_base_s;
+        if (tid == 32) TRACE_SET(1, TRACE_CLOCK() - tr_t0);      // set-up done
     }
 
-    if (warp == 1 || warp == 6) {
+    if (warp >= 1 && mw < nmw) {
         // ---------------------------------------------------------- MMA issuers
-        // Two warps, each responsible for every second accumulator tile: the cost of issuing an
-        // MMA (about 80 cycles) is per warp, and tiles are independent.
-        const int mw = warp == 1 ? 0 : 1;
+        // Warp mw issues the MMAs of tiles mw, mw + nmw, ...
         // The whole warp runs the loop so that the descriptor arithmetic stays in
         // uniform registers; one elected lane issues each MMA and commit.
         const uint32_t idesc = make_idesc(p.BN);
@@ -404,7 +439,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 tac = 0;
                 ++chunk;
             }
+            [[maybe_unused]] const long long twa = TRACE_CLOCK();
             got = mbar_wait(&fullA[sa], (ta / kSlotsA) & 1, abort_flag);
+            if (leader && warp == 1) { TRACE_ADD(2, TRACE_CLOCK() - twa); if (kt == kt_begin) TRACE_SET(3, TRACE_CLOCK() - tr_t0); }
             if (!__all_sync(0xffffffffu, got)) {
                 if (leader) flag_timeout(&abort_s, p.status, 0x200u + sa);
                 ok = false;
@@ -413,7 +450,9 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             const uint32_t a_lo0 = desc_lo(a_base + sa * p.a_slot_bytes, p.a_chunk_bytes);
             for (int cls = 0; cls < ncls_mine; ++cls, ++tb) {
                 const int sb = tb % p.slotsB;
+                [[maybe_unused]] const long long twb = TRACE_CLOCK();
                 got = mbar_wait(&fullB[sb], (tb / p.slotsB) & 1, abort_flag);
+                if (leader && warp == 1) TRACE_ADD(4, TRACE_CLOCK() - twb);
                 if (!__all_sync(0xffffffffu, got)) {
                     if (leader) flag_timeout(&abort_s, p.status, 0x280u + sb);
                     ok = false;
@@ -425,7 +464,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 // this chunk of the K-slice), or, collapsed, the first K-tile (a collapsed tile
                 // belongs to one class only)
                 const uint32_t first = (p.collapse ? tac : (tac | cls)) == 0 ? 0u : 1u;
-                for (int u = mw; u < nunits; u += kMmaWarps) {
+                for (int u = mw; u < nunits; u += nmw) {
                     if (p.collapse && unit_cls[u] != cls) continue;
                     // A tap shifts the start by whole 128-byte rows. The swizzle is a function of
                     // the absolute shared-memory address (TMA wrote the tile that way, slots are
@@ -449,6 +488,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
             __syncwarp();
         }
         if (ok && leader) mma_commit(&done_bar);
+        if (leader && warp == 1) TRACE_SET(5, TRACE_CLOCK() - tr_t0);   // last MMA issued
     }
     __syncwarp();
 
@@ -456,6 +496,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     const int nchunk_k = p.chunk_kt > 0 ? (kt_end - kt_begin + p.chunk_kt - 1) / p.chunk_kt : 1;
     for (int kchunk = 0; warp >= 2 && warp < 6 && kchunk < nchunk_k; ++kchunk) {
         bool ok = mbar_wait(&done_bar, kchunk & 1, abort_flag);
+        if (warp == 2 && lane == 0 && kchunk + 1 == nchunk_k) TRACE_SET(6, TRACE_CLOCK() - tr_t0);   // accumulators complete
         if (!ok) flag_timeout(&abort_s, p.status, 0x300u);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -519,7 +560,20 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
+#ifdef AC_TC2_TRACE
+    if (tid == 0) { TRACE_SET(7, clock64() - tr_t0); TRACE_SET(11, trace_gtime()); TRACE_SET(12, kt_end - kt_begin); TRACE_SET(13, nunits); }
+#endif
 }
+
+#ifdef AC_TC2_TRACE
+}  // namespace
+}  // namespace ac
+extern "C" int ac_debug_read_trace(long long* host_out, int words) {
+    return (int)cudaMemcpyFromSymbol(host_out, ac::g_trace, sizeof(long long) * words);
+}
+namespace ac {
+namespace {
+#endif
 
 // Reduction of the collapsed partial tensor P[slice][co block][ci block][tile][co][ci]:
 //   dW[co][r][s][ci] = sum over classes, sum over K-slices of the tile that tap (r,s) maps to in
@@ -845,6 +899,9 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     {
         constexpr int want = 2;   // at least two gradient slots; two instead of three costs ~10 %
         for (int Ic = 1; Ic <= I; ++Ic) {
+#ifdef AC_TC2_TRACE
+            if (const char* f = getenv("AC_TC2_FORCE_IC")) { if (Ic != atoi(f)) continue; }   // development: try one K-tile height
+#endif
             if (Ic + g.uspan > 256) break;
             if (p.strided_map && (p.c_h * (Ic + g.uspan) > 256 || p.c_w * p.Wzq > 256)) break;
             for (int NB = 1; NB <= (Ic == I ? 16 : 1) && NB <= d.N; ++NB) {
