@@ -862,8 +862,7 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     // K-tile shape: Ic class rows of one image, or NB whole class images (then the gradient
     // tile keeps the input tile's row count per image so that both stay on one flat pitch;
     // the surplus rows are beyond the class's extent and arrive as zeros). Chosen by a cost
-    // model per image: a class tile costs max(MMA time, issue time + fixed turn-around),
-    // measured at about 80 cycles per MMA issued and 400 cycles per tile.
+    // model of the busiest CTA's main loop (below).
     const int U = p.collapse ? p.cu_cap : (p.pair_mode ? pairs.count : up.units);
     const double mma_clk = up.BN >= 128 ? up.BN / 2.0 : 48.0;   // N = 64 is shared-memory-read bound
     p.collapse = 0;
@@ -897,7 +896,7 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     int best_Ic = 0, best_sb = 0, best_NB = 1;
     double best_cost = 1e30, best_eff = 0.0;
     {
-        constexpr int want = 2;   // at least two gradient slots; two instead of three costs ~10 %
+        constexpr int want = 2;   // at least two gradient slots
         for (int Ic = 1; Ic <= I; ++Ic) {
 #ifdef AC_TC2_TRACE
             if (const char* f = getenv("AC_TC2_FORCE_IC")) { if (Ic != atoi(f)) continue; }   // development: try one K-tile height
@@ -916,14 +915,28 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
                 if (sb > kMaxSlotsB) sb = kMaxSlotsB;
                 const int bands = (I + Ic - 1) / Ic;
                 const double tiles_per_image = NB == 1 ? (double)bands : 1.0 / NB;
-                const double mmas = (double)U * (KT / 16);
-                const double tile = mmas * mma_clk > 400.0 + 80.0 * mmas ? mmas * mma_clk : 400.0 + 80.0 * mmas;
+                // Two models of a K-tile's time, both fitted to measurements. Layers with several output
+                // classes: a class tile costs max(MMA time, 400 + 80 cycles per MMA), times 1.1 when only
+                // two gradient slots fit. Layers with ONE class (stride = k) change their input tile with
+                // every gradient tile, and what they pay for is that change: the MMA time plus ~600
+                // cycles per K-tile, never less than the ~2050 cycles of a TMA round trip (the input
+                // ring is two deep), and no penalty for two gradient slots -- so they want tall tiles
+                // (3x3 stride 2 on 56x56 at batch 128: 35.8 us with 4-row tiles, 32.5 us with 6-row ones).
+                const double ks = KT / 16, mmas = (double)U * ks;
+                double ktile;
+                if (p.ncls == 1) {
+                    ktile = mmas * mma_clk + 600.0;
+                    if (ktile < 2050.0) ktile = 2050.0;
+                } else {
+                    const double tile = mmas * mma_clk > 400.0 + 80.0 * mmas ? mmas * mma_clk : 400.0 + 80.0 * mmas;
+                    ktile = p.ncls * tile * (sb < 3 ? 1.1 : 1.0);
+                }
                 // what the slowest CTA does: K-tiles are dealt out whole, so the busiest K-slice
                 // sets the time (448 tiles over 148 slices means 4 for some and 3 for most)
                 const long long kts = NB > 1 ? (d.N + NB - 1) / NB : (long long)d.N * bands;
                 long long spl = kNumSMs / p.groups < 1 ? 1 : kNumSMs / p.groups;
                 if (spl > kts) spl = kts;
-                const double cost = (double)((kts + spl - 1) / spl) * p.ncls * tile * (sb < 3 ? 1.1 : 1.0);
+                const double cost = (double)((kts + spl - 1) / spl) * ktile;
                 if (cost < best_cost * (1.0 - 1e-9)) {
                     best_cost = cost; best_Ic = Ic; best_sb = sb; best_NB = NB;
                     best_eff = (double)d.Ho * d.Wo / (tiles_per_image * p.ncls * KT);
