@@ -986,6 +986,9 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
         // slices than that number needs (896 tiles: 128 slices of 7 finish when 148 slices of 6 or 7
         // do, with fewer partial sums to write and reduce, and leave SMs to other streams)
         const int per_slice = (p.ktiles + splits - 1) / splits;
+#ifdef AC_TC2_TRACE
+        if (!getenv("AC_TC2_NO_TRIM"))
+#endif
         splits = (p.ktiles + per_slice - 1) / per_slice;
     }
     p.splits = splits;

@@ -39,7 +39,9 @@ RESNET50 = [
 BOTTLENECK = [(256, 64, 56, 1, 1, 0, 1), (64, 64, 56, 3, 1, 1, 1), (64, 256, 56, 1, 1, 0, 1), (128, 128, 56, 3, 2, 1, 1)]
 RESNET18_STACK = [(64, 64, 56, 3, 1, 1, 1), (128, 128, 28, 3, 1, 1, 1), (256, 256, 14, 3, 1, 1, 1),
                   (512, 512, 8, 3, 1, 1, 1), (512, 512, 7, 3, 1, 1, 1)]
-WORKLOADS = {"resnet50": (RESNET50, 256), "bottleneck": (BOTTLENECK, 128), "resnet18_stack": (RESNET18_STACK, 64)}
+SWEEP = [(128, 128, 64, 3, 1, 1, 1)]     # the pooling-factor sweep's layer (run it with --k 1, 2, 4, 8)
+WORKLOADS = {"resnet50": (RESNET50, 256), "bottleneck": (BOTTLENECK, 128), "resnet18_stack": (RESNET18_STACK, 64),
+             "sweep": (SWEEP, 256)}
 # ResNet-50 convolutions whose input another convolution reads too (the first block of a stage feeds
 # both conv1 and the downsample projection): that tensor is saved, and compressed, once.
 RESNET50_SHARED_INPUT = {(64, 256, 56, 1, 1): 1, (256, 512, 56, 1, 2): 1, (512, 1024, 28, 1, 2): 1,
@@ -113,6 +115,34 @@ def measure(d, dev, reps, seed_images=2):
     return t_c, t_w
 
 
+def gradient_alignment(layers, N, ks, dtype, layout, dev):
+    """Section 5.2's measure, cos = a.b / (|a| |b|), between the weight gradient from the compressed
+    input (pooling factor k) and the one from the full input (k = 1), per layer, on the synthetic
+    inputs. The paper draws its figure from ImageNet activations after an epoch of training; seeded
+    noise has no spatial correlation for the pooling to preserve, so these values are a lower bound
+    of what smooth activations give, and only their order across layers and k is meaningful."""
+    rows = []
+    for ci, co, H, R, st, pd, cnt in layers:
+        base = api.ConvDesc(N, ci, co, H, H, R, R, (st, st), (pd, pd), 1, dtype, layout)
+        x = synth.to_layout(synth.activation(7, (N, ci, H, H), dtype), layout).to(dev)
+        dy = synth.to_layout(synth.grad_output(7, (N, co, base.Ho, base.Wo), dtype), layout).to(dev)
+        grads = {}
+        for k in [1] + [k for k in ks if k != 1]:
+            d = api.ConvDesc(N, ci, co, H, H, R, R, (st, st), (pd, pd), k, dtype, layout)
+            z = torch.empty(d.z_shape, dtype=d.torch_dtype, device=dev)
+            dw = torch.empty(d.dw_shape, dtype=torch.float32, device=dev)
+            ws = torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)
+            api.ac_compress(d, x, z)
+            api.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws)
+            st_, detail = api.ac_workspace_status(ws)
+            if st_ != 0:
+                raise RuntimeError(f"device status {st_} detail {detail:#x}")
+            grads[k] = dw.double().flatten()
+        ref = grads[1]
+        rows.append(((ci, co, H, R, st), {k: float(torch.dot(g, ref) / (g.norm() * ref.norm())) for k, g in grads.items()}))
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
@@ -124,9 +154,22 @@ def main():
     ap.add_argument("--peaks", default=os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))),
                                                     "MEASURED_PEAKS.json"),
                     help="JSON with hbm_gbs and bf16_tflops measured on this machine")
+    ap.add_argument("--cosine", action="store_true",
+                    help="instead of timing: cosine similarity of the compressed and the k = 1 weight gradient per layer")
     a = ap.parse_args()
     layers, batch = WORKLOADS[a.workload]
     N = a.batch or batch
+    if a.cosine:
+        ks = [2, 4, 8]
+        N = a.batch or 8
+        rows = gradient_alignment(layers, N, ks, a.dtype, a.layout, torch.device("cuda:0"))
+        print(f"# {a.workload}: cosine similarity of dW(k) and dW(1) (Section 5.2), batch {N}, {a.dtype} {a.layout}, "
+              "synthetic inputs (X = max(N(0,1),0), dY ~ N(0,1e-4))")
+        print("| C_in→C_out, H, RxS/stride | " + " | ".join(f"k = {k}" for k in ks) + " |")
+        print("|---|" + "---|" * len(ks))
+        for (ci, co, H, R, st), c in rows:
+            print(f"| {ci}→{co}, {H}², {R}x{R}/{st} | " + " | ".join(f"{c[k]:.3f}" for k in ks) + " |")
+        return
     hbm, tens, src = load_peaks(a.peaks)
     dev = torch.device("cuda:0")
     elt = 2 if a.dtype == "bf16" else 4
