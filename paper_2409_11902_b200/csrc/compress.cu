@@ -331,6 +331,98 @@ compress_generic(const T* x, T* __restrict__ z, T* y, int C, int H, int W, int k
     z[idx] = from_f<T>(acc * (1.0f / (float)((h1 - h0) * (w1 - w0))));
 }
 
+// ---- NHWC, C not a multiple of the vector width but rows of W * C elements that are -----------
+// (a network's 3-channel input). The input rows of RB pooled rows go through shared memory: they are
+// fetched with 16-byte loads that are contiguous across the block (a row of W * C elements is one
+// dense run of bytes, whatever C is), each thread then forms outputs from 2- or 4-byte shared-memory
+// reads, and the pooled rows leave as 16-byte stores again when their length allows it.
+// Grid: x = group of RB pooled rows, y = image. Dynamic shared memory: kh * RB input rows + RB
+// output rows.
+// CC, KK: channel count and (square) pooling factor when known at compile time (0: run-time values),
+// so that the index arithmetic per output has no division and the sums unroll.
+template <typename T, bool RELU, int CC, int KK>
+__global__ void __launch_bounds__(256)
+compress_nhwc_rows(const T* x, T* __restrict__ z, T* y, int C_, int H, int W, int kh_, int kw_, int Hp, int Wp,
+                   int RB, int vec_out) {
+    extern __shared__ __align__(16) unsigned char rows_smem[];
+    pdl_launch_dependents();
+    constexpr int VW = VecTraits<T>::VW;
+    const int C = CC > 0 ? CC : C_, kh = KK > 0 ? KK : kh_, kw = KK > 0 ? KK : kw_;
+    const int row_el = W * C, out_el = Wp * C;
+    const int row_v = row_el / VW;                        // 16-byte vectors per input row
+    T* in = reinterpret_cast<T*>(rows_smem);              // [kh * RB][row_el]
+    T* out = in + (size_t)kh * RB * row_el;               // [RB][out_el]
+    const int p0 = blockIdx.x * RB;
+    const long long n = blockIdx.y;
+    const int h_begin = p0 * kh;
+    const int h_end = min(H, (p0 + RB) * kh);             // input rows [h_begin, h_end) are this block's
+    const int nrows = h_end - h_begin;
+    const T* src = x + (n * H + h_begin) * (long long)row_el;
+    // all of a thread's loads are issued before the first is used
+    for (int v = threadIdx.x; v < nrows * row_v; v += 256) {
+        uint4 raw = load16<!RELU>(src + (size_t)v * VW);
+        if (RELU) {
+            float f[VW];
+            unpack<T, true>(raw, f);                      // raw becomes max(raw, 0)
+            *reinterpret_cast<uint4*>(y + (n * H + h_begin) * (long long)row_el + (size_t)v * VW) = raw;
+        }
+        reinterpret_cast<uint4*>(in)[v] = raw;
+    }
+    __syncthreads();
+    const int prows = min(RB, Hp - p0);
+    for (int r = 0; r < prows; ++r) {
+        const int h0 = (p0 + r) * kh, h1 = min(h0 + kh, H);
+        const T* band = in + (size_t)(h0 - h_begin) * row_el;
+        // consecutive threads, consecutive outputs: their shared-memory reads are about 2 elements apart
+        for (int j = threadIdx.x; j < out_el; j += 256) {
+            const int q = j / C, c = j - q * C;
+            const int w0 = q * kw;
+            const T* cell = band + w0 * C + c;
+            float acc = 0.f;
+            float cnt;
+            if (KK > 0 && h1 - h0 == KK && w0 + KK <= W) {
+#pragma unroll
+                for (int dh = 0; dh < (KK > 0 ? KK : 1); ++dh) {
+                    float row = 0.f;
+#pragma unroll
+                    for (int dw = 0; dw < (KK > 0 ? KK : 1); ++dw) row += to_f(cell[dh * row_el + dw * C]);
+                    acc += row;
+                }
+                cnt = (float)(KK * KK);
+            } else {
+                const int w1 = min(w0 + kw, W);
+                for (int h = h0; h < h1; ++h) {
+                    float row = 0.f;
+                    for (int w = w0; w < w1; ++w) row += to_f(cell[(h - h0) * row_el + (w - w0) * C]);
+                    acc += row;
+                }
+                cnt = (float)((h1 - h0) * (w1 - w0));
+            }
+            const T val = from_f<T>(acc * (1.0f / cnt));
+            if (vec_out) out[r * out_el + j] = val;
+            else z[((n * Hp + p0 + r) * (long long)Wp) * C + j] = val;
+        }
+    }
+    if (!vec_out) return;
+    __syncthreads();
+    uint4* dst = reinterpret_cast<uint4*>(z + ((n * Hp + p0) * (long long)Wp) * C);
+    for (int v = threadIdx.x; v < prows * out_el / VW; v += 256) dst[v] = reinterpret_cast<const uint4*>(out)[v];
+}
+
+// Whether the row kernel takes the problem, and with how many pooled rows per block (0: no).
+template <typename T>
+int rows_per_block(const Dims& d) {
+    constexpr int VW = VecTraits<T>::VW;
+    const long long row_el = (long long)d.W * d.Ci, out_el = (long long)d.Wp * d.Ci;
+    if (d.layout != AC_NHWC || row_el % VW != 0 || d.N > 65535) return 0;
+    const long long per_row = (d.kh * row_el + out_el) * (long long)sizeof(T);      // shared memory per pooled row
+    if (per_row > 40 * 1024) return 0;
+    long long rb = (24 * 1024) / per_row;      // about 24 KB per block (measured best of 4 ... 40 KB on a 3-channel 224 x 224 input)
+    if (rb < 1) rb = 1;
+    if (rb > d.Hp) rb = d.Hp;
+    return (int)rb;
+}
+
 inline unsigned blocks_for(long long total) { return (unsigned)((total + 255) / 256); }
 
 template <typename T, int K, int MODE>
@@ -372,6 +464,27 @@ ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, unsigned char* mas
         else launch_nchw_vec<T, 8, MODE>(d, x, z, y, mask, total, st);
     } else {
         if (MODE == 2) return AC_ERR_UNSUPPORTED;
+        if (const int rb = rows_per_block<T>(d)) {
+            const long long out_el = (long long)d.Wp * d.Ci;
+            const int vec_out = (out_el % VW == 0) ? 1 : 0;     // then every pooled row starts 16-byte aligned
+            const size_t smem = (size_t)rb * (d.kh * (size_t)d.W * d.Ci + out_el) * sizeof(T);
+            dim3 grid((unsigned)((d.Hp + rb - 1) / rb), (unsigned)d.N);
+            const bool k2 = d.kh == 2 && d.kw == 2, c3 = d.Ci == 3;
+            if (c3 && k2)
+                compress_nhwc_rows<T, MODE != 0, 3, 2><<<grid, 256, smem, st>>>(x, z, y, d.Ci, d.H, d.W, d.kh, d.kw, d.Hp,
+                                                                                d.Wp, rb, vec_out);
+            else if (c3)
+                compress_nhwc_rows<T, MODE != 0, 3, 0><<<grid, 256, smem, st>>>(x, z, y, d.Ci, d.H, d.W, d.kh, d.kw, d.Hp,
+                                                                                d.Wp, rb, vec_out);
+            else if (k2)
+                compress_nhwc_rows<T, MODE != 0, 0, 2><<<grid, 256, smem, st>>>(x, z, y, d.Ci, d.H, d.W, d.kh, d.kw, d.Hp,
+                                                                                d.Wp, rb, vec_out);
+            else
+                compress_nhwc_rows<T, MODE != 0, 0, 0><<<grid, 256, smem, st>>>(x, z, y, d.Ci, d.H, d.W, d.kh, d.kw, d.Hp,
+                                                                                d.Wp, rb, vec_out);
+            AC_CUDA_TRY(cudaGetLastError());
+            return AC_OK;
+        }
         compress_generic<T, MODE != 0><<<blocks_for(zt), 256, 0, st>>>(
             x, z, y, d.Ci, d.H, d.W, d.kh, d.kw, d.Hp, d.Wp, d.layout == AC_NHWC, zt);
     }
