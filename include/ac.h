@@ -144,7 +144,9 @@ ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z
  * position reads gathered into a [N*H_o*W_o][taps x C_in] bf16 matrix in the
  * workspace (at most 256 columns, padded to a multiple of 64; taps that read
  * the same element of Z for every position share one column) and run as the
- * equivalent 1x1 problem on the tensor cores. All other problems, and calls
+ * equivalent 1x1 problem on the tensor cores; where the strides are multiples
+ * of k and k divides H and W (a 7x7 stride-2 stem at k = 2) that matrix is
+ * built tile by tile in shared memory instead and needs no workspace. All other problems, and calls
  * whose workspace is smaller than ac_workspace_bytes but at least
  * ac_workspace_bytes_min, use fp32 FMA (or the slower tensor-core kernel) on
  * the operands as they are.
@@ -298,7 +300,12 @@ ac_status ac_conv2d_wgrad_compressed_rect(const ac_conv_desc *desc, int32_t k_h,
  * reports and tests). Returns AC_ERR_INVALID_ARG for an invalid descriptor.
  */
 typedef struct {
-    int32_t tensor_core;     /* 5: bf16 NHWC with fewer than 64 input channels (a 3-channel stem): the
+    int32_t tensor_core;     /* 6: as 5 when taps share columns (both strides multiples of k, k divides H
+                                and W, at most 128 columns, rows of Z a multiple of 16 bytes long): the matrix
+                                is never written to memory; sixteen warps of the kernel build each K-tile
+                                of it in shared memory from a strip of Z rows fetched by TMA, beside the
+                                warp that issues the MMAs (band_rows = whole output rows per K-tile),
+                                5: bf16 NHWC with fewer than 64 input channels (a 3-channel stem): the
                                 inflated, zero-padded values every output position reads are gathered
                                 into a [positions][taps x C_in] matrix in the workspace (one column
                                 per distinct shift of Z instead of per tap when both strides are

@@ -129,7 +129,9 @@ size_t ac_workspace_bytes_min(const ac_conv_desc* desc) {
     Dims d;
     if (make_dims(desc, true, &d) != AC_OK) return 0;
     const WgradPlan p = plan_wgrad(d);
-    return p.path == PATH_STAGED || p.path == PATH_GATHER ? plan_wgrad_unstaged(d).bytes : p.bytes;
+    if (p.path != PATH_STAGED && p.path != PATH_GATHER) return p.bytes;
+    const size_t plain = plan_wgrad_unstaged(d).bytes;      // the path on the operands as they are
+    return plain < p.bytes ? plain : p.bytes;
 }
 
 ac_status ac_compress(const ac_conv_desc* desc, const void* x, void* z, void* y_out, void* stream) {

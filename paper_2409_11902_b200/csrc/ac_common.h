@@ -93,6 +93,12 @@ void plan_gather(const Dims& d, WgradPlan* p);
 void gather_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_gather(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                               float* dw, void* workspace, cudaStream_t stream);
+// the same with the operand matrix built inside the kernel (wgrad_gather_fused.cu): layers whose taps share columns
+bool gather_fused_supported(const Dims& d);
+size_t gather_fused_workspace_bytes(const Dims& d);
+void gather_fused_plan_info(const Dims& d, ac_plan_info* info);
+ac_status launch_wgrad_gather_fused(const Dims& d, const void* z, const void* dy, float* dw, void* workspace,
+                                    cudaStream_t stream);
 size_t tc2_collapsed_workspace_bytes(const Dims& d, int* tiles_collapsed, int* tiles_dense);
 ac_status launch_wgrad_tc2_collapsed(const Dims& d, const void* z, const void* dy, float* dw,
                                      void* workspace, cudaStream_t stream);

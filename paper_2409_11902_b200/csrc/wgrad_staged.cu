@@ -558,9 +558,15 @@ ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z,
     return AC_OK;
 }
 
-bool gather_supported(const Dims& d) { return gather_geom(d).ok; }
+bool gather_supported(const Dims& d) { return gather_fused_supported(d) || gather_geom(d).ok; }
 
 void plan_gather(const Dims& d, WgradPlan* pl) {
+    if (gather_fused_supported(d)) {      // the matrix is built inside the kernel: no staged copy
+        *pl = WgradPlan{};
+        pl->path = PATH_GATHER;
+        pl->bytes = gather_fused_workspace_bytes(d);
+        return;
+    }
     const GatherGeom g = gather_geom(d);
     plan_tc2(g.in, pl);
     pl->path = PATH_GATHER;
@@ -572,6 +578,10 @@ void plan_gather(const Dims& d, WgradPlan* pl) {
 }
 
 void gather_plan_info(const Dims& d, ac_plan_info* info) {
+    if (gather_fused_supported(d)) {
+        gather_fused_plan_info(d, info);
+        return;
+    }
     const GatherGeom g = gather_geom(d);
     tc2_plan_info(g.in, info);
     info->tensor_core = 5;
@@ -579,6 +589,7 @@ void gather_plan_info(const Dims& d, ac_plan_info* info) {
 
 ac_status launch_wgrad_gather(const Dims& d, const WgradPlan& pl, const void* z, const void* dy, float* dw,
                               void* workspace, cudaStream_t stream) {
+    if (gather_fused_supported(d)) return launch_wgrad_gather_fused(d, z, dy, dw, workspace, stream);
     const GatherGeom g = gather_geom(d);
     if (!g.ok) return AC_ERR_UNSUPPORTED;
     char* ws = static_cast<char*>(workspace);

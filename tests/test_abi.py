@@ -189,15 +189,15 @@ def test_few_input_channels_are_gathered_for_the_tensor_cores(ac):
     runs the equivalent 1x1 problem on the output map."""
     def inner(N, cols, co, Ho, Wo):
         return ac.ConvDesc(N, cols, co, Ho, Wo, 1, 1, (1, 1), (0, 0), 1, "bf16", "nhwc")
-    # 7x7, stride 2, pad 3, k = 2, k | H: taps collapse to 4 x 4 shifts -> 48 columns, padded to 64
+    # 7x7, stride 2, pad 3, k = 2, k | H: taps collapse to 4 x 4 shifts -> 48 columns, padded to 64; such layers
+    # have the matrix built inside the kernel (plan code 6): K-tiles of 16 whole output rows of 16 positions, and no
+    # staged copy in the workspace, only the K-slices of the [C_out][64] result
     d = ac.ConvDesc(8, 3, 64, 32, 32, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc")
     i = ac.ac_wgrad_plan_info(d)
-    assert i["tensor_core"] == 5
-    di = inner(8, 64, 64, 16, 16)
-    ii = ac.ac_wgrad_plan_info(di)
-    assert ii["tensor_core"] == 2 and {k: v for k, v in i.items() if k != "tensor_core"} == \
-        {k: v for k, v in ii.items() if k != "tensor_core"}
-    assert ac.ac_workspace_bytes(d) == ac.ac_workspace_bytes(di) + 8 * 16 * 16 * 64 * 2 + 64 * 64 * 4
+    assert i["tensor_core"] == 6 and i["k_tile"] == 256 and i["band_rows"] == 16 and i["block_n"] == 64
+    assert i["splits"] == 8 * 16 // 16 and i["smem_bytes"] <= 227 * 1024 and i["tmem_columns"] == 64
+    assert ac.ac_workspace_bytes(d) == 256 + i["splits"] * 64 * 64 * 4
+    assert ac.ac_workspace_bytes_min(d) <= ac.ac_workspace_bytes(d)
     # an odd map cannot collapse (the partial last block): one column per tap, 147 -> 192
     d = ac.ConvDesc(8, 3, 64, 31, 31, 7, 7, (2, 2), (3, 3), 2, "bf16", "nhwc")
     assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 5

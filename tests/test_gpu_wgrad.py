@@ -419,6 +419,11 @@ FEW_CHANNELS = [
     (1, 1, 64, 9, 9, 3, 3, 1, 0, 3),        # one channel, k = 3, no padding
     (2, 3, 64, 32, 32, 3, 5, 2, 1, 2),      # R != S, collapsed
     (2, 7, 192, 8, 8, 1, 1, 1, 0, 2),       # pointwise
+    (3, 3, 64, 56, 64, 7, 7, 2, 3, 2),      # in-kernel form: 32 positions per row, 4 rows per K-tile
+    (3, 3, 64, 56, 40, 7, 7, 2, 3, 2),      # rows of Z of 120 bytes: not for TMA, staged in the workspace
+    (2, 6, 320, 24, 24, 3, 3, 2, 1, 2),     # in-kernel form, 320 output channels = 5 blocks of 64
+    (2, 8, 256, 16, 48, 5, 5, 2, 2, 2),     # in-kernel form: 3 x 3 shifts x 8 channels = 72 columns -> 128, N = 256
+    (5, 3, 64, 12, 12, 7, 7, 4, 3, 2),      # stride 4 = 2k: two pooled rows per output row, a 3-position row
 ]
 
 
@@ -426,7 +431,12 @@ FEW_CHANNELS = [
 def test_few_input_channels_match_checker(case):
     import paper_2409_11902_b200 as ac
     d = D(*case, "bf16", "nhwc")
-    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 5
+    N, Ci, Co, H, W, R, S, stride, pad, k = case
+    # strides that are multiples of k on a map that k divides: the matrix is built inside the kernel (6);
+    # otherwise it is staged in the workspace (5)
+    # (and rows of Z that are a whole number of 16-byte units long, for the TMA copy of the strip)
+    fused = k > 1 and stride % k == 0 and H % k == 0 and W % k == 0 and ((W // k) * Ci * 2) % 16 == 0
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == (6 if fused else 5)
     err, got, want = wgrad_error_full(d)
     assert err <= 1e-4 <= TOL_DW["bf16"], err     # bf16 products are exact in fp32: summation order only
 
