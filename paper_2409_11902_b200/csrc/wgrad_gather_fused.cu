@@ -320,8 +320,9 @@ __global__ void __launch_bounds__(kGfThreads, 1) wgrad_gather_fused_kernel(const
     if (warp == 1) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
-// dW[co][r][s][ci] = sum over K-slices of slice[co][column of (r, s, ci)], slices in index order
-// (four interleaved running sums).
+// dW[co][r][s][ci] = sum over K-slices of slice[co][column of (r, s, ci)]. One warp per element of dW:
+// lane l adds slices l, l + 32, ... in order, then the 32 running sums are combined by a butterfly
+// (a fixed tree), so the result does not depend on anything but the slices.
 struct GfReduceParams {
     int splits, R, S, Ci, ph, pw, k, u0, v0, nb, Mp;
     long long slice_elems, total;
@@ -330,26 +331,20 @@ struct GfReduceParams {
 __global__ void __launch_bounds__(256) gf_reduce_scatter_kernel(const float* __restrict__ partials, GfReduceParams q,
                                                                 float* __restrict__ dw) {
     pdl_wait();
-    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long i = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (i >= q.total) return;
+    const int lane = threadIdx.x & 31;
     const int row = q.R * q.S * q.Ci;
     const long long co = i / row;
     const int rem = (int)(i - co * row);
     const int t = rem / q.Ci, ci = rem - t * q.Ci, r = t / q.S, s = t - r * q.S;
     const int iu = floor_div_i(r - q.ph, q.k) - q.u0, iv = floor_div_i(s - q.pw, q.k) - q.v0;
     const float* src = partials + co * q.Mp + (iu * q.nb + iv) * q.Ci + ci;
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-    int sp = 0;
-    for (; sp + 4 <= q.splits; sp += 4) {
-        s0 += __ldcs(src + (long long)(sp + 0) * q.slice_elems);
-        s1 += __ldcs(src + (long long)(sp + 1) * q.slice_elems);
-        s2 += __ldcs(src + (long long)(sp + 2) * q.slice_elems);
-        s3 += __ldcs(src + (long long)(sp + 3) * q.slice_elems);
-    }
-    if (sp + 0 < q.splits) s0 += __ldcs(src + (long long)(sp + 0) * q.slice_elems);
-    if (sp + 1 < q.splits) s1 += __ldcs(src + (long long)(sp + 1) * q.slice_elems);
-    if (sp + 2 < q.splits) s2 += __ldcs(src + (long long)(sp + 2) * q.slice_elems);
-    dw[i] = (s0 + s1) + (s2 + s3);
+    float acc = 0.f;
+    for (int sp = lane; sp < q.splits; sp += 32) acc += __ldcs(src + (long long)sp * q.slice_elems);
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+    if (lane == 0) dw[i] = acc;
 }
 
 // ------------------------------------------------------------------ host side
@@ -530,7 +525,7 @@ ac_status launch_wgrad_gather_fused(const Dims& d, const void* z, const void* dy
     GfReduceParams q;
     q.splits = p.splits; q.R = d.R; q.S = d.S; q.Ci = d.Ci; q.ph = d.ph; q.pw = d.pw; q.k = d.k;
     q.u0 = p.u0; q.v0 = p.v0; q.nb = p.nb; q.Mp = p.Mp; q.slice_elems = p.slice_elems; q.total = p.dw_elems;
-    launch_after(gf_reduce_scatter_kernel, dim3((unsigned)((q.total + 255) / 256)), dim3(256), 0, stream,
+    launch_after(gf_reduce_scatter_kernel, dim3((unsigned)((q.total + 7) / 8)), dim3(256), 0, stream,
                  static_cast<const float*>(partials), q, dw);
     AC_CUDA_TRY(cudaGetLastError());
     return AC_OK;
