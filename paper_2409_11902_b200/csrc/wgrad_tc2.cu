@@ -32,7 +32,6 @@
 // is split over CTAs and the partial dW tensors are summed in a fixed order afterwards.
 #include <cuda.h>
 
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -898,9 +897,6 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     {
         constexpr int want = 2;   // at least two gradient slots
         for (int Ic = 1; Ic <= I; ++Ic) {
-#ifdef AC_TC2_TRACE
-            if (const char* f = getenv("AC_TC2_FORCE_IC")) { if (Ic != atoi(f)) continue; }   // development: try one K-tile height
-#endif
             if (Ic + g.uspan > 256) break;
             if (p.strided_map && (p.c_h * (Ic + g.uspan) > 256 || p.c_w * p.Wzq > 256)) break;
             for (int NB = 1; NB <= (Ic == I ? 16 : 1) && NB <= d.N; ++NB) {
@@ -986,9 +982,6 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
         // slices than that number needs (896 tiles: 128 slices of 7 finish when 148 slices of 6 or 7
         // do, with fewer partial sums to write and reduce, and leave SMs to other streams)
         const int per_slice = (p.ktiles + splits - 1) / splits;
-#ifdef AC_TC2_TRACE
-        if (!getenv("AC_TC2_NO_TRIM"))
-#endif
         splits = (p.ktiles + per_slice - 1) / per_slice;
     }
     p.splits = splits;
