@@ -44,7 +44,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads2 = 224;        // warp 0: TMA, warps 1 and 6: MMA (1 owns TMEM), warps 2-5: epilogue (and MMA)
+constexpr int kThreads2 = 256;        // warps 0 and 7: TMA, warps 1 and 6: MMA (1 owns TMEM), warps 2-5: epilogue (and MMA)
+constexpr int kProducers = 2;         // TMA-issuing warps (a third would leave each thread too few registers)
 constexpr int kMaxMmaWarps = 6;       // accumulator tiles are dealt out over up to this many issuing warps
 constexpr int kMaxUnits2 = 8;
 constexpr int kMaxClasses = 64;      // output classes (k/s_h * k/s_w), e.g. k = 8 at stride 1
@@ -233,27 +234,33 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
     const uint32_t a_base = smem_base, b_base = smem_base + kSlotsA * p.a_slot_bytes;
 
 
-    // ---------------------------------------------------------------- TMA producer
-    // Warp 0 issues every copy. The stream of copies is: for each K-tile, the Z halo
-    // tile (one copy per 8-channel plane, one plane per lane so that the planes of a
-    // tile go out as one warp instruction), then one gradient tile per class (one
-    // 64-channel chunk per lane). It is written as a resumable loop so that the first
-    // tiles, which need no free slot, are already in flight while the other warps do
-    // the set-up work below.
-    int pr_kt = kt_begin, pr_ta = 0, pr_cls = -1, pr_tb = 0;
-    auto produce = [&](bool may_wait) {
+    // ---------------------------------------------------------------- TMA producers
+    // The stream of copies is, for each K-tile, the Z halo tile (one 64-channel chunk per lane, so that
+    // the chunks of a tile go out as one warp instruction), then one gradient tile per class (likewise).
+    // Issuing one such instruction takes a warp 650-850 cycles (measured with a stand-alone loop: 650
+    // for one box, +55 for each further lane), whatever the state of the barriers, while a second
+    // warp's copies go out in parallel (two issuing warps: twice the rate). For layers whose tiles
+    // carry little arithmetic (1x1 and stride-2 layers: a K-tile of 1000-2000 cycles of MMAs needs two
+    // to five copies) one warp cannot keep up, so two warps issue. Each SLOT of the two rings belongs
+    // to one producer warp for good: a wait on a slot's barrier tests the parity of its phase, which
+    // is only right for a waiter that has seen every earlier phase of that barrier go by (a warp that
+    // came to the slot two phases early would find the parity it looks for and overwrite a tile in
+    // use). Every warp walks the whole stream in order and issues the copies whose slot is its own;
+    // the MMA warps consume in stream order, so the producers need no order among themselves.
+    const int pw_idx = warp == 0 ? 0 : warp - 6;      // producer warps 0 and 7 -> 0, 1
+    auto produce = [&]() {
         const int nchunk_ld = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);   // 64-channel chunks per variant
         const int nloads = nchunk_ld * p.nvar;
-        while (pr_kt < kt_end) {
-            const int n = p.NB > 1 ? pr_kt * p.NB : pr_kt / p.bands;
-            const int i0 = p.NB > 1 ? 0 : (pr_kt - n * p.bands) * p.Ic;
-            if (pr_cls < 0) {
-                const int sa = pr_ta % kSlotsA;
-                if (pr_ta >= kSlotsA) {
-                    if (!may_wait) return;
+        int tb = 0;
+        for (int t = 0, kt = kt_begin; kt < kt_end; ++t, ++kt) {
+            const int n = p.NB > 1 ? kt * p.NB : kt / p.bands;
+            const int i0 = p.NB > 1 ? 0 : (kt - n * p.bands) * p.Ic;
+            const int sa = t % kSlotsA;
+            if (sa % kProducers == pw_idx) {
+                if (t >= kSlotsA) {
                     [[maybe_unused]] const long long tw = TRACE_CLOCK();
-                    const bool got = mbar_wait(&emptyA[sa], ((pr_ta / kSlotsA) & 1) ^ 1, abort_flag);
-                    if (lane == 0) TRACE_ADD(8, TRACE_CLOCK() - tw);
+                    const bool got = mbar_wait(&emptyA[sa], ((t / kSlotsA) & 1) ^ 1, abort_flag);
+                    if (lane == 0 && warp == 0) TRACE_ADD(8, TRACE_CLOCK() - tw);
                     if (!__all_sync(0xffffffffu, got)) {
                         if (lane == 0) flag_timeout(&abort_s, p.status, 0x100u + sa);
                         return;
@@ -272,14 +279,14 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                     tma_load_4d(a_slot + (vs * p.chunksA + c) * p.a_chunk_bytes, &p.tmA[var], &fullA[sa],
                                 cib0 * p.CB + ch, p.vmin + dv, i0 + p.umin + du, n);
                 }
-                pr_cls = 0;
-            } else {
-                const int sb = pr_tb % p.slotsB;
-                if (pr_tb >= p.slotsB) {
-                    if (!may_wait) return;
+            }
+            for (int cl = 0; cl < ncls_mine; ++cl, ++tb) {
+                const int sb = tb % p.slotsB;
+                if ((sb + kSlotsA) % kProducers != pw_idx) continue;      // offset: the warps with an input slot get fewer
+                if (tb >= p.slotsB) {
                     [[maybe_unused]] const long long tw = TRACE_CLOCK();
-                    const bool got = mbar_wait(&emptyB[sb], ((pr_tb / p.slotsB) & 1) ^ 1, abort_flag);
-                    if (lane == 0) TRACE_ADD(9, TRACE_CLOCK() - tw);
+                    const bool got = mbar_wait(&emptyB[sb], ((tb / p.slotsB) & 1) ^ 1, abort_flag);
+                    if (lane == 0 && warp == 0) TRACE_ADD(9, TRACE_CLOCK() - tw);
                     if (!__all_sync(0xffffffffu, got)) {
                         if (lane == 0) flag_timeout(&abort_s, p.status, 0x180u + sb);
                         return;
@@ -289,7 +296,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 __syncwarp();
                 const uint32_t b_slot = b_base + sb * p.b_slot_bytes;
                 if (lane < p.nchunks) {
-                    const int cls_id = cls0 + pr_cls;
+                    const int cls_id = cls0 + cl;
                     if (p.strided_map) {
                         // one map over dY, traversed with strides (c_w, c_h): the class is the start
                         const int a = cls_id / p.c_w, b = cls_id - a * p.c_w;
@@ -300,8 +307,6 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                                     co0 + 64 * lane, 0, i0, n);
                     }
                 }
-                ++pr_tb;
-                if (++pr_cls == ncls_mine) { pr_cls = -1; ++pr_kt; ++pr_ta; }
             }
         }
     };
@@ -327,8 +332,10 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         __syncwarp();
         // The barriers are ready, which is all the other warps need from this one: it reports in
         // at the set-up barrier without waiting there and goes straight on to issuing copies
-        // (issuing the first round of them takes about 3 us; the first tile lands long before).
+        // (the first tile lands long before the set-up is over). The other producer warp waits
+        // for nothing but this (barrier 3).
         __threadfence_block();
+        bar_arrive(3, kProducers * 32);
         bar_arrive(1, kThreads2);
         // Everything up to here touched no global memory and may have run while the kernel before
         // this one in the stream (the compress kernel that writes Z, say) was still finishing.
@@ -336,16 +343,21 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         // The status block starts clean: CTA 0 resets it here, long before any wait of this launch
         // can run out (a wait gives up only after 2^32 cycles).
         if (blockIdx.x == 0 && lane == 0 && !p.keep_status) { p.status[0] = 0u; p.status[1] = 0u; }
-        produce(true);
+        produce();
         if (lane == 0) TRACE_SET(10, TRACE_CLOCK() - tr_t0);    // producer done
+    } else if (warp >= 7) {
+        bar_sync(3, kProducers * 32);      // the mbarriers exist
+        bar_arrive(1, kThreads2);
+        pdl_wait();
+        produce();
     }
     // Everything the MMAs may read but no copy ever writes must be finite (it only
     // ever meets zeros of the other operand, or feeds accumulator rows that are
     // discarded): the cells behind the last row of each input plane, the planes of
     // the unused upper 64 rows when CB = 64, and the gradient rows behind the tile.
     if (warp == 1) tmem_alloc(&tmem_base_s, p.tmem_cols);   // about 0.6 us, beside the zero fill
-    if (warp >= 2) {
-        constexpr int kZeroWarps = kThreads2 / 32 - 2;
+    if (warp >= 2 && warp <= 6) {
+        constexpr int kZeroWarps = 5;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         const int chunks_real = p.pair_mode ? p.ncopies : ncib * (p.CB / 64);
         const int units16 = (int)(p.a_chunk_bytes / 16), written = p.NB * p.rowsA * p.Wzq * 8;
@@ -363,7 +375,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         }
         fence_proxy_async_smem();
     }
-    if (warp >= 1) {
+    if (warp >= 1 && warp <= 6) {
         if (p.collapse && tid == 32) {
             // tile u = number cj0 + u: find its class and its shift inside the class
             int base = 0, u = 0;
@@ -379,7 +391,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 base += cnt;
             }
         }
-        for (int t2 = tid - 32; !p.collapse && t2 < p.ncls * kMaxUnits2; t2 += kThreads2 - 32) {
+        for (int t2 = tid - 32; !p.collapse && t2 < p.ncls * kMaxUnits2; t2 += 192) {
             const int cls = t2 / kMaxUnits2, u = t2 % kMaxUnits2;
             uint32_t off = 0;
             if (p.pair_mode) {
@@ -401,7 +413,7 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
         }
     }
     uint32_t tmem_base = 0;
-    if (warp >= 1) {
+    if (warp >= 1 && warp <= 6) {
         tc_fence_before();
         bar_sync(1, kThreads2);
         tc_fence_after();
