@@ -31,7 +31,10 @@ namespace {
 using namespace tc;
 
 constexpr int kGfBuilders = 512;    // a multiple of the 16-byte chunks per row of G (8 or 16): a thread's chunk never changes
-constexpr int kGfThreads = 64 + kGfBuilders;     // warp 0: TMA, warp 1: MMA + tensor memory, the rest: build, then drain
+constexpr int kGfStripWarp = 2 + kGfBuilders / 32;     // the last warp
+// warp 0: dY tiles by TMA, warp 1: MMA + tensor memory, the builders (build, then drain), last warp: Z strips by
+// TMA. Issuing a tensor copy holds a warp for several hundred cycles, so the two streams have a warp each.
+constexpr int kGfThreads = 64 + kGfBuilders + 32;
 constexpr int kGfSlotsA = 3;
 constexpr int kGfMaxSlotsB = 4;
 constexpr int kGfSlotsS = 4;        // ring of Z strips
@@ -108,7 +111,7 @@ __global__ void __launch_bounds__(kGfThreads, 1) wgrad_gather_fused_kernel(const
         }
     } else if (warp == 1) {
         tmem_alloc(&tmem_base_s, p.tmem_cols);
-    } else {
+    } else if (warp < kGfStripWarp) {
         // Everything the MMAs read but nobody writes later must be zero: the input tiles' cells behind
         // the last position and the padding columns of their rows, and the gradient tiles' cells
         // behind the box that TMA fills.
@@ -133,6 +136,23 @@ __global__ void __launch_bounds__(kGfThreads, 1) wgrad_gather_fused_kernel(const
     if (warp == 0) {
         // ------------------------------------------------------------ dY tiles by TMA
         for (int kt = kt_begin, i = 0; kt < kt_end; ++kt, ++i) {
+            const int sb = i % p.slotsB;
+            if (i >= p.slotsB) {
+                const bool got = mbar_wait(&emptyB[sb], ((i / p.slotsB) & 1) ^ 1, abort_flag);
+                if (!__all_sync(0xffffffffu, got)) {
+                    if (lane == 0) gf_timeout(&abort_s, p.status, 0x480u + sb);
+                    break;
+                }
+            }
+            if (lane == 0) mbar_arrive_expect_tx(&fullB[sb], (uint32_t)p.nchunks * p.b_box_bytes);
+            __syncwarp();
+            if (lane < p.nchunks)
+                tma_load_3d(b_base + sb * p.b_slot_bytes + lane * p.b_chunk_bytes, &p.tmB, &fullB[sb], co0 + 64 * lane,
+                            0, kt * p.RB);
+        }
+    } else if (warp == kGfStripWarp) {
+        // ------------------------------------------------------------ Z strips by TMA
+        for (int kt = kt_begin, i = 0; kt < kt_end; ++kt, ++i) {
             // the strip of Z this K-tile reads: rows rb .. rb + nz - 1 of image n, from element x0 on; rows and
             // elements outside Z arrive as zeros (the convolution's padding)
             const int ss = i % kGfSlotsS;
@@ -148,19 +168,7 @@ __global__ void __launch_bounds__(kGfThreads, 1) wgrad_gather_fused_kernel(const
                 mbar_arrive_expect_tx(&fullS[ss], p.strip_box_bytes);
                 tma_load_3d(s_base + ss * p.strip_bytes, &p.tmZ, &fullS[ss], p.x0 / 2, ho * p.mh + p.u0, n);
             }
-            const int sb = i % p.slotsB;
-            if (i >= p.slotsB) {
-                const bool got = mbar_wait(&emptyB[sb], ((i / p.slotsB) & 1) ^ 1, abort_flag);
-                if (!__all_sync(0xffffffffu, got)) {
-                    if (lane == 0) gf_timeout(&abort_s, p.status, 0x480u + sb);
-                    break;
-                }
-            }
-            if (lane == 0) mbar_arrive_expect_tx(&fullB[sb], (uint32_t)p.nchunks * p.b_box_bytes);
             __syncwarp();
-            if (lane < p.nchunks)
-                tma_load_3d(b_base + sb * p.b_slot_bytes + lane * p.b_chunk_bytes, &p.tmB, &fullB[sb], co0 + 64 * lane,
-                            0, kt * p.RB);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
