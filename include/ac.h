@@ -300,7 +300,15 @@ ac_status ac_conv2d_wgrad_compressed_rect(const ac_conv_desc *desc, int32_t k_h,
  * reports and tests). Returns AC_ERR_INVALID_ARG for an invalid descriptor.
  */
 typedef struct {
-    int32_t tensor_core;     /* 6: as 5 when taps share columns (both strides multiples of k, k divides H
+    int32_t tensor_core;     /* 7: bf16 NHWC problems with partial pooling blocks next to the padding (an
+                                odd map, padded taps) on which kernel 2 is expected to be slower reading
+                                Z than reading the inflated map (3x3 on 7x7 at k = 2: four differently
+                                zeroed copies of a 5x5-cell tile per image and class), or cannot keep its
+                                tile copies in shared memory at all: the inflated map Xt is written to the
+                                workspace (|X| bytes) and kernel 2 runs on it with k = 1 (described by
+                                the other fields); with a workspace of ac_workspace_bytes_min() bytes
+                                the kernel reads Z itself where it can,
+                                6: as 5 when taps share columns (both strides multiples of k, k divides H
                                 and W, at most 128 columns, rows of Z a multiple of 16 bytes long): the matrix
                                 is never written to memory; sixteen warps of the kernel build each K-tile
                                 of it in shared memory from a strip of Z rows fetched by TMA, beside the

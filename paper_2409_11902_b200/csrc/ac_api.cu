@@ -77,6 +77,11 @@ void record_timing_hook(int which, cudaStream_t stream) {
 
 // The plan for a caller whose workspace has no room for staged operand copies.
 WgradPlan plan_wgrad_unstaged(const Dims& d) {
+    if (tc2_supported(d, nullptr)) {
+        WgradPlan p{};
+        plan_tc2(d, &p);
+        return p;
+    }
     if (tc_supported(d)) {
         WgradPlan p{};
         p.path = PATH_TC;
@@ -89,7 +94,7 @@ WgradPlan plan_wgrad_unstaged(const Dims& d) {
 WgradPlan plan_wgrad(const Dims& d) {
     if (tc2_supported(d, nullptr)) {
         WgradPlan p{};
-        plan_tc2(d, &p);
+        if (staged_inflate_preferred(d)) plan_staged(d, &p); else plan_tc2(d, &p);
         return p;
     }
     if (staged_supported(d)) {
@@ -275,7 +280,7 @@ ac_status ac_wgrad_plan_info(const ac_conv_desc* desc, ac_plan_info* info) {
     if (st != AC_OK) return st;
     *info = ac_plan_info{};
     if (tc2_supported(d, nullptr)) {
-        tc2_plan_info(d, info);
+        if (staged_inflate_preferred(d)) staged_plan_info(d, info); else tc2_plan_info(d, info);
         return AC_OK;
     }
     if (staged_supported(d)) {

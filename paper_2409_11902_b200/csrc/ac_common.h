@@ -81,8 +81,12 @@ void tc2_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_tc2(const Dims& d, const WgradPlan& p, const void* z, const void* dy,
                            float* dw, void* workspace, cudaStream_t stream, bool keep_status = false);
 int tc2_chain_length(const Dims& d);
+double tc2_cost_cycles(const Dims& d, int* tile_copies);
 // fp32 and/or NCHW inputs staged for the TMA-fed kernel (wgrad_staged.cu)
 bool staged_supported(const Dims& d);
+// bf16 NHWC problems the TMA-fed kernel takes directly but that run faster on an inflated copy of Z
+// (small odd maps with padding); true: plan and launch them as staged problems
+bool staged_inflate_preferred(const Dims& d);
 void plan_staged(const Dims& d, WgradPlan* p);
 void staged_plan_info(const Dims& d, ac_plan_info* info);
 ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& p, const void* z, const void* dy,

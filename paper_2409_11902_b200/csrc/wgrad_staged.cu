@@ -35,11 +35,35 @@
 //    EVERY position, so taps with equal (u, v) have equal columns: G then keeps one column per distinct
 //    (u, v, channel) (7x7, stride 2, pad 3, k = 2: 16 shifts instead of 49 taps; 48 columns instead of
 //    147, a third of the bytes written and read) and the last pass copies each column to all its taps.
+//
+//  * Small odd maps with padding (3x3 on 7x7 at k = 2; bf16 NHWC). The kernel reads Z directly here too, but
+//    pays for it: every output class multiplies a whole tile of Z cells (its halo included) into every tap,
+//    a pooled row or column that covers a partial block has to be kept in up to four differently zeroed
+//    copies, and on a 4x4 grid of cells the halo and the rounding of a K-tile to 16 cells outweigh what the
+//    compression saves (128 cell products per image and tap where the inflated 7x7 map needs 64). When the
+//    kernel's cost model says so, the staging pass writes the inflated map Xt (a few MB for such layers) and
+//    the kernel runs on it with k = 1. The same is done for large odd maps with padding whose tile copies do
+//    not fit the shared memory at all.
 #include "ac_common.h"
 #include "tc_units.h"
 
 namespace ac {
 namespace {
+
+// Xt[n][h][w][c] = Z[n][h / kh][w / kw][c], bf16 NHWC, eight channels (16 bytes) per thread
+__global__ void __launch_bounds__(256)
+inflate_nhwc_kernel(const uint4* __restrict__ z, uint4* __restrict__ xt, int H, int W, int Hp, int Wp, int C8, int kh,
+                    int kw, long long total) {
+    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (i >= total) return;
+    const int c = (int)(i % C8);
+    long long r = i / C8;
+    const int w = (int)(r % W);
+    r /= W;
+    const int h = (int)(r % H);
+    const long long n = r / H;
+    xt[i] = __ldg(z + ((n * Hp + h / kh) * Wp + w / kw) * C8 + c);
+}
 
 __device__ __forceinline__ uint32_t pack_bf2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -416,9 +440,36 @@ struct Inner {
     Dims a, b;
 };
 
+// The dense problem on the inflated map, when the cost model expects it to beat the kernel's own reading of Z
+// by a margin (the inflation pass is charged at the copy bandwidth plus a launch), or when the kernel cannot
+// read Z itself (large odd maps with padding, whose four tile copies do not fit the shared memory).
+bool inflate_problem(const Dims& d, Dims* out) {
+    if (d.dtype != AC_BF16 || d.layout != AC_NHWC || (d.kh == 1 && d.kw == 1) || d.max_chain != 0) return false;
+    int copies = 0;
+    const double direct = tc2_cost_cycles(d, &copies);      // negative: the kernel cannot read this Z at all
+    if (direct >= 0.0 && copies < 2) return false;
+    Dims in = d;
+    in.k = in.kh = in.kw = 1;
+    in.Hp = d.H;
+    in.Wp = d.W;
+    if (in.z_elems() >= (1ll << 40) || (in.z_elems() / 8 + 255) / 256 >= (1ll << 31)) return false;
+    const double inflated = tc2_cost_cycles(in, nullptr);
+    if (inflated < 0.0) return false;
+    const double pass = 6000.0 + 2.0 * (double)(d.z_elems() + in.z_elems()) * 2.9e-4;     // cycles: launch + bytes at ~3.4 KB/clk
+    if (direct >= 0.0 && inflated + pass >= 0.85 * direct) return false;
+    *out = in;
+    return true;
+}
+
 bool inner_problem(const Dims& d, Inner* out) {
     const bool split = d.dtype == AC_F32, transpose = d.layout == AC_NCHW;
-    if (!split && !transpose) return false;                 // the kernel reads these itself
+    if (!split && !transpose) {
+        // the kernel reads these itself, and does unless the inflated map is the faster way
+        if (!inflate_problem(d, &out->a)) return false;
+        out->b = out->a;
+        out->b.N = 0;
+        return true;
+    }
     if (transpose) {
         if (d.Ci % 64 != 0 || d.Co % 64 != 0 || d.N > 65535) return false;
         if ((long long)d.Hp * d.Wp >= (1ll << 31) || (long long)d.Ho * d.Wo >= (1ll << 31)) return false;
@@ -486,6 +537,11 @@ bool staged_supported(const Dims& d) {
     return inner_problem(d, &in);
 }
 
+bool staged_inflate_preferred(const Dims& d) {
+    Dims in;
+    return inflate_problem(d, &in);
+}
+
 void plan_staged(const Dims& d, WgradPlan* pl) {
     Inner in;
     inner_problem(d, &in);
@@ -496,10 +552,11 @@ void plan_staged(const Dims& d, WgradPlan* pl) {
         if (pb.bytes > pl->bytes) pl->bytes = pb.bytes;     // the launches use the partial sums' room in turn
     }
     const long long blocks = d.dtype == AC_F32 ? 6 : 1;
+    const bool inflate = d.dtype == AC_BF16 && d.layout == AC_NHWC;      // Xt in place of Z, dY as it is
     pl->path = PATH_STAGED;
     pl->st_off_z = up256(pl->bytes);
-    pl->st_off_dy = pl->st_off_z + up256((size_t)(d.z_elems() * blocks) * 2);
-    pl->st_off_dw = pl->st_off_dy + up256((size_t)(d.dy_elems() * blocks) * 2);
+    pl->st_off_dy = pl->st_off_z + up256((size_t)((inflate ? in.a.z_elems() : d.z_elems()) * blocks) * 2);
+    pl->st_off_dw = pl->st_off_dy + (inflate ? 0 : up256((size_t)(d.dy_elems() * blocks) * 2));
     pl->st_off_small = pl->st_off_dw + (d.layout == AC_NCHW ? up256((size_t)d.dw_elems() * 4) : 0);
     pl->bytes = pl->st_off_small + (in.b.N > 0 ? up256((size_t)d.dw_elems() * 4) : 0);
 }
@@ -508,7 +565,7 @@ void staged_plan_info(const Dims& d, ac_plan_info* info) {
     Inner in;
     inner_problem(d, &in);
     tc2_plan_info(in.a, info);
-    info->tensor_core = in.b.N > 0 ? 4 : 3;
+    info->tensor_core = d.dtype == AC_BF16 && d.layout == AC_NHWC ? 7 : (in.b.N > 0 ? 4 : 3);
 }
 
 ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z, const void* dy,
@@ -519,6 +576,14 @@ ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z,
     char* z_st = ws + pl.st_off_z;
     char* dy_st = ws + pl.st_off_dy;
     ac_status st = AC_OK;
+    if (d.dtype == AC_BF16 && d.layout == AC_NHWC) {
+        const long long total = in.a.z_elems() / 8;
+        inflate_nhwc_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+            static_cast<const uint4*>(z), reinterpret_cast<uint4*>(z_st), d.H, d.W, d.Hp, d.Wp, d.Ci / 8, d.kh, d.kw,
+            total);
+        AC_CUDA_TRY(cudaGetLastError());
+        return launch_wgrad_tc2(in.a, pl, z_st, dy, dw, workspace, stream);
+    }
     if (d.layout == AC_NCHW) {
         if (d.dtype == AC_F32)
             st = stage_nchw<float, true>((const float*)z, (const float*)dy, z_st, dy_st, d, stream);

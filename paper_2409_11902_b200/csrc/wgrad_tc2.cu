@@ -1215,6 +1215,15 @@ int tc2_chain_length(const Dims& d) {
     return (g.p.ktiles + g.p.splits - 1) / g.p.splits * g.p.ncls * g.p.ksteps;
 }
 
+// The cost model's main-loop time (cycles) of the busiest CTA, and how many copies of the input tile
+// the plan keeps (more than one: partial pooling blocks next to the padding). Negative: not supported.
+double tc2_cost_cycles(const Dims& d, int* tile_copies) {
+    const Tc2Geom g = make_geom2(d);
+    if (!g.ok) return -1.0;
+    if (tile_copies) *tile_copies = g.p.nvar;
+    return g.cta_cycles;
+}
+
 // Collapsed form: same dW, fewer MMAs (see Tc2Params::collapse). 0 bytes / AC_ERR_UNSUPPORTED when the
 // problem has nothing to collapse or the TMA-fed kernel does not take it.
 size_t tc2_collapsed_workspace_bytes(const Dims& d, int* tiles_collapsed, int* tiles_dense) {

@@ -120,7 +120,10 @@ def test_plan_info_respects_hardware_limits(ac):
         for k in (1, 2, 4, 8):
             d = ac.ConvDesc(N, ci, co, H, W, R, S, (st, st), (pd, pd), k, "bf16", "nhwc")
             i = ac.ac_wgrad_plan_info(d)
-            assert i["tensor_core"] in (1, 2), d
+            assert i["tensor_core"] in (1, 2, 7), d
+            inflated = i["tensor_core"] == 7     # the TMA-fed kernel on an inflated copy of Z kept in the workspace
+            if inflated:
+                assert k > 1 and (H % k or W % k) and pd > 0
             assert 2 <= i["stages"] <= 8
             assert i["smem_bytes"] <= 227 * 1024
             assert i["tmem_columns"] in (32, 64, 128, 256, 512)
@@ -130,13 +133,16 @@ def test_plan_info_respects_hardware_limits(ac):
                 assert i["k_tile"] >= i["band_rows"] * i["row_pitch"]
                 assert i["row_pitch"] >= d.Wo
             else:   # per class: (band_rows / c_h) class rows of row_pitch >= Wo / c_w positions
-                c_h, c_w = k // st, k // st
+                c_h = c_w = 1 if inflated else k // st
                 assert i["phases"] == c_h * c_w <= 64
                 assert i["k_tile"] >= (i["band_rows"] // c_h) * i["row_pitch"]
                 assert i["row_pitch"] >= -(-d.Wo // c_w)
             assert 1 <= i["splits"] <= d.N * -(-d.Ho // i["band_rows"])
             assert i["ctas"] == i["splits"] * i["groups"]
             want = 256 + (i["splits"] * 4 * co * ci * R * S if i["splits"] > 1 else 0)
+            if inflated:
+                want = -(-want // 256) * 256 + -(-N * H * W * ci * 2 // 256) * 256
+                assert ac.ac_workspace_bytes_min(d) <= want
             assert ac.ac_workspace_bytes(d) == want
     # 64 input channels, 3x3, k = 2: the nine taps pair up into five accumulator tiles in one CTA
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 64, 64, 56, 56, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
@@ -144,9 +150,12 @@ def test_plan_info_respects_hardware_limits(ac):
     # k = 8 at stride 1: 64 output classes, still the TMA-fed kernel
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(256, 128, 128, 64, 64, 3, 3, (1, 1), (1, 1), 8, "bf16", "nhwc"))
     assert (i["tensor_core"], i["phases"]) == (2, 64)
-    # a map that k does not divide (partial pooling blocks) is still taken by the TMA-fed kernel
+    # a small map that k does not divide, with padding (partial pooling blocks that taps read past): the
+    # TMA-fed kernel runs on the inflated map; without padding, or on a larger map, it reads Z itself
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 512, 512, 7, 7, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
-    assert i["tensor_core"] == 2
+    assert (i["tensor_core"], i["phases"]) == (7, 1)
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 128, 128, 29, 29, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
+    assert (i["tensor_core"], i["phases"]) == (2, 4)
     # ... and a 1x1 layer without padding never reads the padding rows inside the partial last block,
     # so it needs no second copy of the tile: same tiles as on the 8x8 map
     i7, i8 = (ac.ac_wgrad_plan_info(ac.ConvDesc(256, 512, 2048, h, h, 1, 1, (1, 1), (0, 0), 2, "bf16", "nhwc"))

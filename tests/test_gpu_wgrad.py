@@ -454,3 +454,30 @@ def test_few_input_channels_small_workspace_and_full_size_stem():
     # the ResNet stem at its own map size
     err, _ = wgrad_error_sampled(D(8, 3, 64, 224, 224, 7, 7, 2, 3, 2, "bf16", "nhwc"), n_samples=256)
     assert err <= 1e-4, err
+
+
+# Small odd maps with padding: the TMA-fed kernel runs on an inflated copy of Z (plan code 7) where its cost
+# model expects that to beat reading Z directly; the result is the same weight gradient.
+ODD_MAPS_INFLATED = [
+    # N, Ci, Co, H, W, R, S, stride, pad, k
+    (24, 512, 512, 7, 7, 3, 3, 1, 1, 2),      # the last ResNet stage's 3x3 layers
+    (64, 256, 512, 7, 9, 3, 3, 1, 1, 2),      # H != W
+    (12, 512, 256, 7, 7, 3, 3, 1, 1, 4),      # k = 4: blocks of 4 and 3 rows and columns
+    (16, 384, 320, 9, 9, 3, 3, 1, 1, 2),      # 320 output channels = 5 blocks of 64
+    (8, 64, 64, 55, 55, 3, 3, 1, 1, 2),       # a large odd map with 64 channels
+    (3, 64, 128, 28, 28, 3, 3, 1, 1, 8),      # k = 8 on a 28 x 28 map: half a block at the edge
+    (5, 128, 64, 7, 7, 3, 3, 1, 1, 4),
+]
+
+
+@pytest.mark.parametrize("case", ODD_MAPS_INFLATED)
+def test_small_odd_maps_run_on_the_inflated_copy(case):
+    import paper_2409_11902_b200 as ac
+    d = D(*case, "bf16", "nhwc")
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 7
+    z, dy = make_wgrad_inputs(d)
+    # with the full workspace (inflated copy), and with the smallest one (the kernel reads Z itself)
+    for nbytes in sorted({ac.ac_workspace_bytes_min(d), ac.ac_workspace_bytes(d)}):
+        got = run_wgrad(d, z, dy, nbytes=nbytes)
+        err = sampled_check(d, got, z, dy, n_samples=512)
+        assert err <= 1e-4, (nbytes, err)
