@@ -146,3 +146,30 @@ def test_rect_full_size_sampled_on_the_tensor_cores():
     idx = stratified_entries(d, 256, seed=4)
     want = oracle.wgrad_compressed_entries(synth.to_f64(z), synth.to_f64(dy), H, H, 3, 3, (1, 1), (1, 1), k, idx)
     assert_dw_close(got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]], want, "bf16")
+
+
+def test_rect_block_on_the_inflated_route():
+    """A small odd map with padding and a 4 x 2 block: the kernel runs on the inflated copy of Z (the
+    workspace holds it beside the partial sums); stratified entries against the checker."""
+    import torch
+    import oracle
+    import paper_2409_11902_b200 as ac
+    from helpers import stratified_entries
+    from paper_2409_11902_b200 import synth
+    N, C, H, k = 24, 512, 7, (4, 2)
+    d = D(N, C, C, H, H, 3, 3, (1, 1), (1, 1), "bf16", "nhwc")
+    full = ac.ac_workspace_bytes_rect(d, *k)
+    assert (full - 256) % (4 * C * C * 9) == N * H * H * C * 2      # K-slices of dW, then the inflated map
+    x = synth.activation(6, (N, C, H, H), "bf16")
+    z = synth.to_storage(oracle.pool(synth.to_f64(x), k), "bf16")
+    dy = synth.grad_output(6, (N, C, H, H), "bf16")
+    zd, dyd = synth.to_layout(z, "nhwc").cuda(), synth.to_layout(dy, "nhwc").cuda()
+    idx = stratified_entries(d, 256, seed=6)
+    want = oracle.wgrad_compressed_entries(synth.to_f64(z), synth.to_f64(dy), H, H, 3, 3, (1, 1), (1, 1), k, idx)
+    ws = torch.empty(full, dtype=torch.uint8, device="cuda")
+    dw = torch.full(d.dw_shape, float("nan"), device="cuda")
+    ac.ac_conv2d_wgrad_compressed_rect(d, k[0], k[1], zd, dyd, dw, ws, full)
+    assert ac.ac_workspace_status(ws)[0] == 0
+    got = dw.double().cpu().numpy().transpose(0, 3, 1, 2)
+    assert np.isfinite(got).all()
+    assert_dw_close(got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]], want, "bf16")
