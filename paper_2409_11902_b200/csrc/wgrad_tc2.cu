@@ -9,8 +9,8 @@
 // ho = 2i + a, wo = 2j + b (one "class" (a,b) of the four parity classes) tap
 // (r,s) reads Z[i + u][j + v] with u = floor((a - ph + r)/2), v = floor((b - pw
 // + s)/2): a constant shift of the COMPACT Z tile. In general, when the strides
-// divide k and k divides H and W, the outputs split into (k/sh)*(k/sw) classes
-// and each (class, tap) pair is a shift (u,v) of Z. Zero padding falls out of
+// divide k, the outputs split into (k/sh)*(k/sw) classes and each (class, tap)
+// pair is a shift (u,v) of Z. Zero padding falls out of
 // the tile bounds: x < 0 or x >= H  <=>  z < 0 or z >= H/k.
 //
 // Per K-tile (a band of class rows of one image, or several whole class images of a small map):
@@ -26,10 +26,15 @@
 //              with element strides), same swizzle, rows past the class's extent
 //              zero-filled by TMA.
 //   Both use the same flat row pitch Wzq, which is what makes a tap a pure shift.
-// Warp 0 issues the TMA copies (one chunk per lane), warps 1 and 6 issue tcgen05.mma (each
-// every second accumulator tile, one elected lane), warps 2-5 drain the accumulators from
-// tensor memory. Every CTA keeps all the accumulator tiles that fit its 512 TMEM columns; K
-// is split over CTAs and the partial dW tensors are summed in a fixed order afterwards.
+// Warps 0 and 7 issue the TMA copies (one chunk per lane; each ring slot belongs to one of the two
+// warps), warps 1-6 issue tcgen05.mma (each its own accumulator tiles, one elected lane), warps 2-5
+// then drain the accumulators from tensor memory. Every CTA keeps all the accumulator tiles that fit
+// its 512 TMEM columns; K is split over CTAs and the partial dW tensors are summed in a fixed order
+// afterwards.
+//
+// A stride that is a multiple m of k (k = 1 at stride 2) has one class, and output row i reads Z row
+// m*i + u through tap row r (u = floor((r - ph)/k)): row i + floor(u/m) of the phase plane u mod m of Z.
+// The planes the taps use are fetched through strided tensor-map views and kept as the tile's copies.
 #include <cuda.h>
 
 #include <cstring>
@@ -66,6 +71,7 @@ struct Tc2Params {
     int keep_status;   // 1: a launch earlier in the same call owns the status block; do not reset it
     int Ci, Co, R, S, sh, sw, ph, pw, kh, kw;   // pooling block kh x kw (square in the paper: kh = kw = k)
     int c_h, c_w, ncls;
+    int mh, mw;        // stride / pooling block where the stride is the larger one (phase planes of Z, below), else 1
     int umin, vmin;
     int Wzq, Ic, bands, KT, ksteps, rowsA;
     int NB, rowsB;   // images per K-tile (> 1 only when a tile is a whole class image) and dY rows per image
@@ -78,6 +84,10 @@ struct Tc2Params {
     // x in [k*(Hp-1), H) but a tap may also reach the padding rows x in [H, k*Hp), which must read
     // 0. A (class, tap) pair whose x falls in that second range at the last Z row is served from a
     // copy of the tile fetched through a tensor map that ends one row (column) earlier.
+    // When the stride is a multiple m of the pooling block (k = 1 at stride 2: the uncompressed gradient of a
+    // strided layer), output row i reads, through tap row r, Z row m*i + u_r with u_r = floor((r - pad) / k):
+    // row i + floor(u_r / m) of the PHASE PLANE u_r mod m of Z (every m-th row from that phase on). The planes a
+    // layer's taps use take the place of the variants (phase row * 2 + phase column; no partial blocks then).
     int nvar, var_slot[4], rho_h, rho_w;   // variants in use, variant -> position in the slot, H % k, W % k
     int Hp, Wp, Ho, Wo;                    // pooled and output map sizes (which pairs need a variant)
     long long dw_elems;
@@ -116,6 +126,17 @@ __host__ __device__ inline bool reads_padding_in_partial_block(int s, int a, int
     const int num = k * (Hp - 1) + rem + pad - r;      // s * ho of the candidate
     if (num < 0 || num % s != 0) return false;
     return num / s < Ho;
+}
+
+// Shift and phase plane of output class coordinate `a` through tap coordinate r: the Z coordinate read is
+// (k/s classes) i + shift, or (stride a multiple m of k, one class) m*i + u = plane (u mod m), coordinate
+// i + floor(u / m).
+__host__ __device__ inline int tap_shift(int s, int a, int pad, int r, int k, int m, int* phase) {
+    const int u = floor_div_i(s * a - pad + r, k);
+    if (m <= 1) { *phase = 0; return u; }
+    const int q = floor_div_i(u, m);
+    *phase = u - q * m;
+    return q;
 }
 
 // Distinct Z shifts of output class `cls`: rows u0 .. u0+nU-1, columns v0 .. v0+nV-1
@@ -400,11 +421,13 @@ __global__ void __launch_bounds__(kThreads2, 1) wgrad_tc2_kernel(const __grid_co
                 const int cl = u / ntap, t = u - cl * ntap;
                 const int tap = tap0 + t, r = tap / p.S, sx = tap - r * p.S;
                 const int a = cls / p.c_w, b = cls - a * p.c_w;
-                const int uu = floor_div_i(p.sh * a - p.ph + r, p.kh) - p.umin;
-                const int vv = floor_div_i(p.sw * b - p.pw + sx, p.kw) - p.vmin;
-                // which copy of the tile: the one without the partial last row / column of Z if this
-                // (class, tap) reaches past H / W there
-                const int var = (reads_padding_in_partial_block(p.sh, a, p.ph, r, p.kh, p.Hp, p.rho_h, p.Ho) ? 2 : 0) +
+                int fh, fw;
+                const int uu = tap_shift(p.sh, a, p.ph, r, p.kh, p.mh, &fh) - p.umin;
+                const int vv = tap_shift(p.sw, b, p.pw, sx, p.kw, p.mw, &fw) - p.vmin;
+                // which copy of the tile: the phase plane of Z this tap reads (stride a multiple of k), else
+                // the one without the partial last row / column of Z if this (class, tap) reaches past H / W there
+                const int var = p.mh > 1 || p.mw > 1 ? fh * 2 + fw :
+                                (reads_padding_in_partial_block(p.sh, a, p.ph, r, p.kh, p.Hp, p.rho_h, p.Ho) ? 2 : 0) +
                                 (reads_padding_in_partial_block(p.sw, b, p.pw, sx, p.kw, p.Wp, p.rho_w, p.Wo) ? 1 : 0);
                 off = (uint32_t)(p.var_slot[var] * p.chunksA + cl * (p.CB / 64)) * p.a_chunk_bytes +
                       (uint32_t)(uu * p.Wzq + vv) * 128u;
@@ -805,11 +828,16 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     Tc2Params& p = g.p;
     g.ok = false;
     if (d.dtype != AC_BF16 || d.layout != AC_NHWC) return g;
-    if (d.kh % d.sh != 0 || d.kw % d.sw != 0) return g;    // class rows advance Z by exactly one row
+    // class rows advance Z by exactly one row: s | k (k/s classes), or k | s (one class, s/k phase planes of Z)
+    if ((d.kh % d.sh != 0 && d.sh % d.kh != 0) || (d.kw % d.sw != 0 && d.sw % d.kw != 0)) return g;
+    p.mh = d.sh % d.kh == 0 ? d.sh / d.kh : 1;
+    p.mw = d.sw % d.kw == 0 ? d.sw / d.kw : 1;
+    const bool planes = p.mh > 1 || p.mw > 1;
+    if (planes && (collapse || p.mh > 2 || p.mw > 2 || d.H % d.kh != 0 || d.W % d.kw != 0)) return g;
     if (d.R * d.S > 64 || d.R > 16 || d.S > 16) return g;
     const UnitPlan up = plan_units(d.Ci, d.Co, d.R * d.S, kMaxUnits2, fill_rectangles, bn_cap);
     if (!up.ok) return g;
-    p.c_h = d.kh / d.sh; p.c_w = d.kw / d.sw;
+    p.c_h = d.kh % d.sh == 0 ? d.kh / d.sh : 1; p.c_w = d.kw % d.sw == 0 ? d.kw / d.sw : 1;
     p.ncls = p.c_h * p.c_w;
     if (p.ncls > kMaxClasses) return g;
     p.strided_map = p.ncls > kMaxClassMaps ? 1 : 0;
@@ -818,14 +846,19 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     p.kh = d.kh; p.kw = d.kw;
     p.dw_elems = d.dw_elems();
     int umin = 1 << 30, umax = -(1 << 30), vmin = 1 << 30, vmax = -(1 << 30);
+    bool phase_h[2] = {false, false}, phase_w[2] = {false, false};
     for (int a = 0; a < p.c_h; ++a)
         for (int r = 0; r < d.R; ++r) {
-            const int u = floor_div_i(d.sh * a - d.ph + r, d.kh);
+            int ph_;
+            const int u = tap_shift(d.sh, a, d.ph, r, d.kh, p.mh, &ph_);
+            phase_h[ph_] = true;
             umin = u < umin ? u : umin; umax = u > umax ? u : umax;
         }
     for (int b = 0; b < p.c_w; ++b)
         for (int s = 0; s < d.S; ++s) {
-            const int v = floor_div_i(d.sw * b - d.pw + s, d.kw);
+            int ph_;
+            const int v = tap_shift(d.sw, b, d.pw, s, d.kw, p.mw, &ph_);
+            phase_w[ph_] = true;
             vmin = v < vmin ? v : vmin; vmax = v > vmax ? v : vmax;
         }
     p.umin = umin; p.vmin = vmin;
@@ -848,6 +881,13 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
         for (int r = 0; r < d.R; ++r)
             for (int b = 0; b < p.c_w; ++b)
                 for (int s_ = 0; s_ < d.S; ++s_) {
+                    if (planes) {
+                        int fh, fw;
+                        tap_shift(d.sh, a, d.ph, r, d.kh, p.mh, &fh);
+                        tap_shift(d.sw, b, d.pw, s_, d.kw, p.mw, &fw);
+                        var_used[fh * 2 + fw] = true;
+                        continue;
+                    }
                     var_used[(reads_padding_in_partial_block(d.sh, a, d.ph, r, d.kh, d.Hp, p.rho_h, d.Ho) ? 2 : 0) +
                              (reads_padding_in_partial_block(d.sw, b, d.pw, s_, d.kw, d.Wp, p.rho_w, d.Wo) ? 1 : 0)] = true;
                 }
@@ -855,9 +895,13 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     for (int v = 0; v < 4; ++v) p.var_slot[v] = var_used[v] ? p.nvar++ : -1;
     if ((var_used[2] || var_used[3]) && d.Hp < 2) return g;
     if ((var_used[1] || var_used[3]) && d.Wp < 2) return g;
+    // extent of the (largest) plane a line of the tile comes from, and whether a plane one shorter is in use too
+    const int ext_h = (d.Hp + p.mh - 1) / p.mh, ext_w = (d.Wp + p.mw - 1) / p.mw;
+    const bool short_h = planes ? (phase_h[1] && (d.Hp - 1 + p.mh - 1) / p.mh < ext_h) : (var_used[2] || var_used[3]);
+    const bool short_w = planes ? (phase_w[1] && (d.Wp - 1 + p.mw - 1) / p.mw < ext_w) : (var_used[1] || var_used[3]);
     PairPlan pairs{};
     p.pair_mode = 0;
-    if (kEnablePairs && !collapse && p.nvar == 1 && d.Ci == 64 && plan_pairs(d, p.c_h, p.c_w, umin, vmin, g.uspan, g.vspan, &pairs) &&
+    if (kEnablePairs && !collapse && !planes && p.nvar == 1 && d.Ci == 64 && plan_pairs(d, p.c_h, p.c_w, umin, vmin, g.uspan, g.vspan, &pairs) &&
         pairs.count * up.BN <= 512) {
         p.pair_mode = 1;
         p.pu_count = pairs.count;
@@ -901,8 +945,8 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
         p.slice_elems = (long long)up.ncob * up.ncib_total * total * up.BN * up.CB;
     }
     if (!p.pair_mode) {
-        p.Wzq = min_flat_pitch(Jc, vmin, vmax, d.Wp, var_used[1] || var_used[3]);
-        rows_whole = min_flat_pitch(I, umin, umax, d.Hp, var_used[2] || var_used[3]);
+        p.Wzq = min_flat_pitch(Jc, vmin, vmax, ext_w, short_w);
+        rows_whole = min_flat_pitch(I, umin, umax, ext_h, short_h);
     }
     int best_Ic = 0, best_sb = 0, best_NB = 1;
     double best_cost = 1e30, best_eff = 0.0;
@@ -1129,13 +1173,24 @@ static ac_status launch_tc2_any(const Dims& d, bool collapse, const void* z, con
         if (p.var_slot[var] < 0) continue;
         // Z viewed as (Ci, Wp, Hp, N); one copy brings 64 channels of a (rows x Wzq) window.
         // Variants 1-3 end one column and/or one row early: the partial last block reads as zero.
-        const cuuint64_t dims[4] = {(cuuint64_t)d.Ci, (cuuint64_t)(d.Wp - (var & 1)),
-                                    (cuuint64_t)(d.Hp - (var >> 1)), (cuuint64_t)d.N};
-        const cuuint64_t strides[3] = {(cuuint64_t)d.Ci * 2, (cuuint64_t)d.Wp * d.Ci * 2,
-                                       (cuuint64_t)d.Hp * d.Wp * d.Ci * 2};
+        cuuint64_t dims[4] = {(cuuint64_t)d.Ci, (cuuint64_t)(d.Wp - (var & 1)),
+                              (cuuint64_t)(d.Hp - (var >> 1)), (cuuint64_t)d.N};
+        cuuint64_t strides[3] = {(cuuint64_t)d.Ci * 2, (cuuint64_t)d.Wp * d.Ci * 2,
+                                 (cuuint64_t)d.Hp * d.Wp * d.Ci * 2};
+        const char* zbase = static_cast<const char*>(z);
+        if (p.mh > 1 || p.mw > 1) {
+            // phase plane (fh, fw): rows fh, fh + mh, ... and columns fw, fw + mw, ... of Z
+            const int fh = var >> 1, fw = var & 1;
+            if (fh >= p.mh || fw >= p.mw || fh >= d.Hp || fw >= d.Wp) return AC_ERR_UNSUPPORTED;
+            dims[1] = (cuuint64_t)((d.Wp - fw + p.mw - 1) / p.mw);
+            dims[2] = (cuuint64_t)((d.Hp - fh + p.mh - 1) / p.mh);
+            strides[0] = (cuuint64_t)p.mw * d.Ci * 2;
+            strides[1] = (cuuint64_t)p.mh * d.Wp * d.Ci * 2;
+            zbase += ((size_t)fh * d.Wp + fw) * d.Ci * 2;
+        }
         const cuuint32_t box[4] = {64, (cuuint32_t)p.Wzq, (cuuint32_t)p.rowsA, (cuuint32_t)p.NB};
         const cuuint32_t es[4] = {1, 1, 1, 1};
-        if (enc(&p.tmA[var], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(z), dims, strides, box, es,
+        if (enc(&p.tmA[var], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<char*>(zbase), dims, strides, box, es,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return AC_ERR_CUDA;

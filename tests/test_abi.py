@@ -133,7 +133,7 @@ def test_plan_info_respects_hardware_limits(ac):
                 assert i["k_tile"] >= i["band_rows"] * i["row_pitch"]
                 assert i["row_pitch"] >= d.Wo
             else:   # per class: (band_rows / c_h) class rows of row_pitch >= Wo / c_w positions
-                c_h = c_w = 1 if inflated else k // st
+                c_h = c_w = 1 if inflated else max(1, k // st)     # a stride above k: one class, phase planes of Z
                 assert i["phases"] == c_h * c_w <= 64
                 assert i["k_tile"] >= (i["band_rows"] // c_h) * i["row_pitch"]
                 assert i["row_pitch"] >= -(-d.Wo // c_w)
@@ -161,8 +161,13 @@ def test_plan_info_respects_hardware_limits(ac):
     i7, i8 = (ac.ac_wgrad_plan_info(ac.ConvDesc(256, 512, 2048, h, h, 1, 1, (1, 1), (0, 0), 2, "bf16", "nhwc"))
               for h in (7, 8))
     assert all(i7[f] == i8[f] for f in ("k_tile", "stages", "smem_bytes", "a_cells", "row_pitch", "ctas"))
-    # a stride that does not divide k goes to the producer-fed tensor-core kernel
+    # a stride that is a multiple of k (k = 1 at stride 2): one class reading phase planes of Z, the TMA-fed kernel
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 28, 28, 3, 3, (2, 2), (1, 1), 1, "bf16", "nhwc"))
+    assert (i["tensor_core"], i["phases"]) == (2, 1)
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 28, 28, 3, 3, (2, 2), (1, 1), 3, "bf16", "nhwc"))
+    assert i["tensor_core"] == 7      # k = 3 at stride 2: the same kernel on the inflated map (k = 1 at stride 2)
+    # what is left to the producer-fed tensor-core kernel: phase planes whose tiles do not fit the shared memory
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(8, 128, 128, 64, 64, 5, 5, (2, 2), (0, 0), 1, "bf16", "nhwc"))
     assert i["tensor_core"] == 1
     # shapes the tensor-core kernel does not take go to the fp32-ALU kernel
     for d in (ac.ConvDesc(8, 24, 64, 32, 32, 3, 3, (1, 1), (1, 1), 2, "f32", "nchw"),

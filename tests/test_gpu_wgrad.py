@@ -481,3 +481,32 @@ def test_small_odd_maps_run_on_the_inflated_copy(case):
         got = run_wgrad(d, z, dy, nbytes=nbytes)
         err = sampled_check(d, got, z, dy, n_samples=512)
         assert err <= 1e-4, (nbytes, err)
+
+
+# A stride that is a multiple of the pooling block (k = 1 at stride 2: the uncompressed gradient of a strided
+# layer): one output class whose taps read phase planes of Z, still the TMA-fed kernel.
+STRIDE_ABOVE_K = [
+    # N, Ci, Co, H, W, R, S, stride, pad, k, dtype, layout, plan code
+    (4, 128, 128, 28, 28, 3, 3, 2, 1, 1, "bf16", "nhwc", 2),
+    (4, 64, 128, 30, 30, 3, 3, 2, 1, 1, "bf16", "nhwc", 2),
+    (4, 64, 64, 29, 31, 3, 3, 2, 1, 1, "bf16", "nhwc", 2),       # odd map: planes of different extents
+    (4, 128, 256, 28, 28, 1, 1, 2, 0, 1, "bf16", "nhwc", 2),     # the downsample projection: one plane, one tap
+    (3, 64, 64, 32, 32, 7, 7, 2, 3, 1, "bf16", "nhwc", 2),
+    (4, 64, 64, 24, 24, 5, 5, 2, 2, 1, "bf16", "nhwc", 2),
+    (4, 64, 64, 32, 32, 3, 3, 4, 1, 2, "bf16", "nhwc", 2),       # stride 4 at k = 2
+    (3, 64, 128, 12, 20, 3, 3, (2, 1), (1, 1), 1, "bf16", "nhwc", 2),
+    (4, 128, 128, 28, 28, 3, 3, 2, 1, 3, "bf16", "nhwc", 7),     # k = 3 at stride 2: inflated, then as above
+    (4, 64, 64, 28, 28, 3, 3, 2, 1, 1, "f32", "nhwc", 3),        # staged operands on the same plan
+    (4, 64, 128, 28, 28, 3, 3, 2, 1, 1, "bf16", "nchw", 3),
+]
+
+
+@pytest.mark.parametrize("case", STRIDE_ABOVE_K)
+def test_stride_above_k_matches_checker(case):
+    import paper_2409_11902_b200 as ac
+    N, Ci, Co, H, W, R, S, stride, pad, k, dtype, layout, code = case
+    pair = lambda v: v if isinstance(v, tuple) else (v, v)
+    d = ac.ConvDesc(N, Ci, Co, H, W, R, S, pair(stride), pair(pad), k, dtype, layout)
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] in ((code,) if code != 3 else (3, 4))
+    err, got, want = wgrad_error_full(d)
+    assert err <= TOL_DW[dtype], err
