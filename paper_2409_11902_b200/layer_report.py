@@ -115,6 +115,58 @@ def measure(d, dev, reps, seed_images=2):
     return t_c, t_w
 
 
+def overlapped_wgrads(layers, N, k, dtype, layout, dev, nstreams, seed_images=2):
+    """Microseconds for the weight gradients of ALL the workload's convolutions (every repeat of a shape
+    its own dW and workspace), last layer first, dealt round-robin to `nstreams` streams inside one
+    captured graph: what a training step that runs independent weight gradients side by side sees."""
+    inst = []
+    for ci, co, H, R, st, pd, cnt in layers:
+        d = api.ConvDesc(N, ci, co, H, H, R, R, (st, st), (pd, pd), k, dtype, layout)
+        nb = min(N, seed_images)
+        rep = (-(-N // nb), 1, 1, 1)
+        x = synth.to_layout(synth.activation(0, (nb, ci, H, H), dtype), layout).to(dev).repeat(rep)[:N].contiguous()
+        dy = synth.to_layout(synth.grad_output(0, (nb, co, d.Ho, d.Wo), dtype), layout).to(dev).repeat(rep)[:N].contiguous()
+        z = torch.empty(d.z_shape, dtype=d.torch_dtype, device=dev)
+        api.ac_compress(d, x, z)
+        del x
+        for _ in range(cnt):
+            inst.append((d, z, dy, torch.empty(d.dw_shape, dtype=torch.float32, device=dev),
+                         torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)))
+    inst.reverse()
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(device=dev) for _ in range(nstreams)]
+
+    def enqueue():
+        main = torch.cuda.current_stream()
+        for s_ in streams:
+            s_.wait_stream(main)
+        for i, (d, z, dy, dw, ws) in enumerate(inst):
+            with torch.cuda.stream(streams[i % nstreams]):
+                api.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws)
+        for s_ in streams:
+            main.wait_stream(s_)
+
+    enqueue()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        enqueue()
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 5
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    for d, z, dy, dw, ws in inst:
+        st, detail = api.ac_workspace_status(ws)
+        if st != 0:
+            raise RuntimeError(f"device status {st} detail {detail:#x}")
+    return e0.elapsed_time(e1) * 1e3 / reps, len(inst), sum(i[0].flops for i in inst)
+
+
 def gradient_alignment(layers, N, ks, dtype, layout, dev):
     """Section 5.2's measure, cos = a.b / (|a| |b|), between the weight gradient from the compressed
     input (pooling factor k) and the one from the full input (k = 1), per layer, on the synthetic
@@ -154,6 +206,8 @@ def main():
     ap.add_argument("--peaks", default=os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))),
                                                     "MEASURED_PEAKS.json"),
                     help="JSON with hbm_gbs and bf16_tflops measured on this machine")
+    ap.add_argument("--streams", type=int, default=0,
+                    help="instead of the per-layer table: all weight gradients of the workload in one graph on this many streams")
     ap.add_argument("--cosine", action="store_true",
                     help="instead of timing: cosine similarity of the compressed and the k = 1 weight gradient per layer")
     a = ap.parse_args()
@@ -173,6 +227,12 @@ def main():
     hbm, tens, src = load_peaks(a.peaks)
     dev = torch.device("cuda:0")
     elt = 2 if a.dtype == "bf16" else 4
+    if a.streams > 0:
+        us, n, fl = overlapped_wgrads(layers, N, a.k, a.dtype, a.layout, dev, a.streams)
+        print(f"# {a.workload}, batch {N}, {a.dtype} {a.layout}, k = {a.k}: the {n} weight gradients as one graph on "
+              f"{a.streams} stream(s): {us:.0f} us = {fl / us / 1e6:.0f} TFLOP/s dense-equivalent "
+              f"({fl / us / 1e6 / tens:.2f} of the {src} tensor peak {tens:.0f})")
+        return
     print(f"# {a.workload}, batch {N}, {a.dtype} {a.layout}, k = {a.k}; denominators ({src}): "
           f"{hbm:.0f} GB/s HBM copy, {tens:.0f} TFLOP/s bf16 burst")
     print("| C_in→C_out, H, RxS/stride | × | path | X MiB | Z MiB | compress µs | GB/s | of HBM | wgrad µs | TFLOP/s "
