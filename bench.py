@@ -441,9 +441,13 @@ def run_ours(args):
         sl = descs(SECONDARY)
         shost = [host_inputs(d, seed=50 + li, n_images=SEED_IMAGES) for li, (_, d) in enumerate(sl)]
         swl = Workload(ac, sl, shost, N_SETS_SECONDARY, dev)
+        # the four layers run side by side on four streams: each plans for its share of the SMs
+        budget = max(1, 148 // len(sl))
+        ac.ac_set_sm_budget(budget)
         for it in range(3):
             swl.step(it)
         sgraphs = swl.step_graphs(concurrent=True)
+        ac.ac_set_sm_budget(0)
         n_sec = max(args.steps, 200)
         t0.record(stream)
         for it in range(n_sec):
@@ -456,7 +460,8 @@ def run_ours(args):
         s_fl = sum(d.flops for _, d in sl)
         secondary = {
             "workload": SECONDARY_WORKLOAD, "ms_per_step": s_ms, "step_tflops": s_fl / s_ms / 1e9,
-            "schedule": "one CUDA graph per buffer set, every layer's chain on a stream of its own",
+            "schedule": "one CUDA graph per buffer set, every layer's chain on a stream of its own, weight gradients "
+                        f"planned for {budget} SMs each (ac_set_sm_budget); per_layer: each layer alone on the whole GPU",
             "l2": f"inputs rotated over {N_SETS_SECONDARY} buffer sets ({N_SETS_SECONDARY * swl.set_bytes / 1e6:.0f} MB, L2 is 126 MB)",
             "per_layer": [{k: p[k] for k in ("layer", "compress_us", "compress_gbs", "wgrad_call_us",
                                              "wgrad_call_tflops", "splits", "ctas")} for p in s_layers]}

@@ -11,5 +11,5 @@ from .api import (  # noqa: F401
     ac_conv2d_wgrad_compressed_static, ac_collapsed_workspace_bytes,
     ac_conv2d_wgrad_compressed_collapsed,
     ac_host_step_arena_bytes, ac_workspace_bytes_rect, ac_compress_rect, ac_conv2d_wgrad_compressed_rect,
-    ac_selftest_bounded_wait, ac_set_kernel_timing_events, ac_wgrad_plan_info, ac_workspace_bytes, ac_workspace_bytes_min, ac_workspace_status, status_string,
+    ac_selftest_bounded_wait, ac_set_kernel_timing_events, ac_set_sm_budget, ac_get_sm_budget, ac_wgrad_plan_info, ac_workspace_bytes, ac_workspace_bytes_min, ac_workspace_status, status_string,
 )

@@ -76,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.ac_conv2d_wgrad_compressed_accumulate.argtypes = [dp, vp, vp, ctypes.c_float, vp, vp, sz, vp]
         L.ac_set_kernel_timing_events.restype = ctypes.c_int
         L.ac_set_kernel_timing_events.argtypes = [vp, vp]
+        L.ac_set_sm_budget.restype = ctypes.c_int
+        L.ac_set_sm_budget.argtypes = [ctypes.c_int32]
+        L.ac_get_sm_budget.restype = ctypes.c_int32
+        L.ac_get_sm_budget.argtypes = []
         L.ac_workspace_status.restype = ctypes.c_int
         L.ac_workspace_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
         L.ac_host_step_arena_bytes.restype = sz
@@ -237,6 +241,17 @@ def ac_set_kernel_timing_events(before=None, after=None) -> None:
     st = lib().ac_set_kernel_timing_events(raw(before), raw(after))
     if st != AC_OK:
         raise AcError(st, "ac_set_kernel_timing_events")
+
+
+def ac_set_sm_budget(sms: int) -> None:
+    """SMs the calling thread's weight-gradient plans may count on (0: the whole GPU); see ac.h."""
+    st = lib().ac_set_sm_budget(int(sms))
+    if st != AC_OK:
+        raise AcError(st, "ac_set_sm_budget")
+
+
+def ac_get_sm_budget() -> int:
+    return int(lib().ac_get_sm_budget())
 
 
 def ac_workspace_status(workspace, stream=None):

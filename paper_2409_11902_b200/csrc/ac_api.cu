@@ -3,6 +3,10 @@
 
 namespace ac {
 
+namespace {
+thread_local int g_sm_budget = kNumSMs;
+}
+
 ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o, int k_h, int k_w) {
     if (!d || !o) return AC_ERR_INVALID_ARG;
     *o = Dims{};   // plans are cached by the bytes of this struct
@@ -15,6 +19,7 @@ ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o, int k_h, int
     o->kh = rect ? k_h : d->k; o->kw = rect ? k_w : d->k; o->k = o->kh;
     o->dtype = d->dtype; o->layout = d->layout;
     o->elt = d->dtype == AC_F32 ? 4 : 2;
+    o->sms = g_sm_budget;
     o->Hp = (d->H + o->kh - 1) / o->kh;
     o->Wp = (d->W + o->kw - 1) / o->kw;
     o->Co = 1; o->R = 1; o->S = 1; o->sh = 1; o->sw = 1; o->ph = 0; o->pw = 0;
@@ -121,6 +126,14 @@ WgradPlan plan_wgrad(const Dims& d) {
 using namespace ac;
 
 extern "C" {
+
+ac_status ac_set_sm_budget(int32_t sms) {
+    if (sms < 0) return AC_ERR_INVALID_ARG;
+    g_sm_budget = sms == 0 || sms > kNumSMs ? kNumSMs : sms;
+    return AC_OK;
+}
+
+int32_t ac_get_sm_budget(void) { return g_sm_budget; }
 
 size_t ac_workspace_bytes(const ac_conv_desc* desc) { return ac_workspace_bytes_rect(desc, 0, 0); }
 

@@ -26,6 +26,9 @@ struct Dims {
     // accumulator with truncation, a bias that grows with the length of the chain; bf16 results
     // (bound 1e-2) never notice, fp32 results assembled from bf16 terms (bound 1e-5) do.
     int max_chain;
+    // SMs a weight-gradient plan may count on (ac_set_sm_budget; kNumSMs unless the caller runs several
+    // weight gradients side by side): the tensor-core paths launch about this many CTAs, one per SM.
+    int sms;
     long long x_elems() const { return (long long)N * Ci * H * W; }
     long long z_elems() const { return (long long)N * Ci * Hp * Wp; }
     long long dy_elems() const { return (long long)N * Co * Ho * Wo; }

@@ -434,7 +434,8 @@ GfGeom gf_geom(const Dims& d) {
     const long long ktiles = (long long)d.N * d.Ho / p.RB;
     if (ktiles >= (1ll << 30)) return g;
     p.ktiles = (int)ktiles;
-    int splits = kNumSMs / p.groups;
+    int splits = d.sms / p.groups;
+    if (splits < 1) splits = 1;
     if (splits > p.ktiles) splits = p.ktiles;
     const int per_slice = (p.ktiles + splits - 1) / splits;
     p.splits = (p.ktiles + per_slice - 1) / per_slice;

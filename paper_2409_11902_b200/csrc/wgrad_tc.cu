@@ -386,7 +386,7 @@ TcGeom make_geom(const Dims& d) {
     p.ktiles = (int)ktiles;
     p.stages = best_stages;
     if (p.stages > p.ktiles) p.stages = p.ktiles < 2 ? 2 : p.ktiles;
-    int splits = kNumSMs / p.groups;
+    int splits = d.sms / p.groups;
     if (splits < 1) splits = 1;
     if (splits > p.ktiles) splits = p.ktiles;
     p.splits = splits;

@@ -986,7 +986,7 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
                 // what the slowest CTA does: K-tiles are dealt out whole, so the busiest K-slice
                 // sets the time (448 tiles over 148 slices means 4 for some and 3 for most)
                 const long long kts = NB > 1 ? (d.N + NB - 1) / NB : (long long)d.N * bands;
-                long long spl = kNumSMs / p.groups < 1 ? 1 : kNumSMs / p.groups;
+                long long spl = d.sms / p.groups < 1 ? 1 : d.sms / p.groups;
                 if (spl > kts) spl = kts;
                 const double cost = (double)((kts + spl - 1) / spl) * ktile;
                 if (cost < best_cost * (1.0 - 1e-9)) {
@@ -1030,7 +1030,7 @@ Tc2Geom build_geom2_with(const Dims& d, bool collapse, bool fill_rectangles, int
     const long long ktiles = p.NB > 1 ? (d.N + p.NB - 1) / p.NB : (long long)d.N * p.bands;
     if (ktiles >= (1ll << 30)) return g;
     p.ktiles = (int)ktiles;
-    int splits = kNumSMs / p.groups;
+    int splits = d.sms / p.groups;
     if (splits < 1) splits = 1;
     if (splits > p.ktiles) splits = p.ktiles;
     {

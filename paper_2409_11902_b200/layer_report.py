@@ -115,7 +115,7 @@ def measure(d, dev, reps, seed_images=2):
     return t_c, t_w
 
 
-def overlapped_wgrads(layers, N, k, dtype, layout, dev, nstreams, seed_images=2):
+def overlapped_wgrads(layers, N, k, dtype, layout, dev, nstreams, budget=0, seed_images=2):
     """Microseconds for the weight gradients of ALL the workload's convolutions (every repeat of a shape
     its own dW and workspace), last layer first, dealt round-robin to `nstreams` streams inside one
     captured graph: what a training step that runs independent weight gradients side by side sees."""
@@ -129,9 +129,11 @@ def overlapped_wgrads(layers, N, k, dtype, layout, dev, nstreams, seed_images=2)
         z = torch.empty(d.z_shape, dtype=d.torch_dtype, device=dev)
         api.ac_compress(d, x, z)
         del x
+        b = budget
+        api.ac_set_sm_budget(b)
         for _ in range(cnt):
             inst.append((d, z, dy, torch.empty(d.dw_shape, dtype=torch.float32, device=dev),
-                         torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)))
+                         torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dev), b))
     inst.reverse()
     torch.cuda.synchronize()
     streams = [torch.cuda.Stream(device=dev) for _ in range(nstreams)]
@@ -140,9 +142,11 @@ def overlapped_wgrads(layers, N, k, dtype, layout, dev, nstreams, seed_images=2)
         main = torch.cuda.current_stream()
         for s_ in streams:
             s_.wait_stream(main)
-        for i, (d, z, dy, dw, ws) in enumerate(inst):
+        for i, (d, z, dy, dw, ws, b) in enumerate(inst):
+            api.ac_set_sm_budget(b)
             with torch.cuda.stream(streams[i % nstreams]):
                 api.ac_conv2d_wgrad_compressed(d, z, dy, dw, ws)
+        api.ac_set_sm_budget(0)
         for s_ in streams:
             main.wait_stream(s_)
 
@@ -160,7 +164,7 @@ def overlapped_wgrads(layers, N, k, dtype, layout, dev, nstreams, seed_images=2)
         g.replay()
     e1.record()
     torch.cuda.synchronize()
-    for d, z, dy, dw, ws in inst:
+    for d, z, dy, dw, ws, b in inst:
         st, detail = api.ac_workspace_status(ws)
         if st != 0:
             raise RuntimeError(f"device status {st} detail {detail:#x}")
@@ -208,6 +212,8 @@ def main():
                     help="JSON with hbm_gbs and bf16_tflops measured on this machine")
     ap.add_argument("--streams", type=int, default=0,
                     help="instead of the per-layer table: all weight gradients of the workload in one graph on this many streams")
+    ap.add_argument("--sm-budget", type=int, default=0,
+                    help="with --streams: SMs each weight gradient plans for (ac_set_sm_budget; 0: the whole GPU)")
     ap.add_argument("--cosine", action="store_true",
                     help="instead of timing: cosine similarity of the compressed and the k = 1 weight gradient per layer")
     a = ap.parse_args()
@@ -228,9 +234,9 @@ def main():
     dev = torch.device("cuda:0")
     elt = 2 if a.dtype == "bf16" else 4
     if a.streams > 0:
-        us, n, fl = overlapped_wgrads(layers, N, a.k, a.dtype, a.layout, dev, a.streams)
+        us, n, fl = overlapped_wgrads(layers, N, a.k, a.dtype, a.layout, dev, a.streams, a.sm_budget)
         print(f"# {a.workload}, batch {N}, {a.dtype} {a.layout}, k = {a.k}: the {n} weight gradients as one graph on "
-              f"{a.streams} stream(s): {us:.0f} us = {fl / us / 1e6:.0f} TFLOP/s dense-equivalent "
+              f"{a.streams} stream(s), each planned for {a.sm_budget or 148} SMs: {us:.0f} us = {fl / us / 1e6:.0f} TFLOP/s dense-equivalent "
               f"({fl / us / 1e6 / tens:.2f} of the {src} tensor peak {tens:.0f})")
         return
     print(f"# {a.workload}, batch {N}, {a.dtype} {a.layout}, k = {a.k}; denominators ({src}): "

@@ -273,3 +273,31 @@ def test_rect_entry_points_validate_the_block(ac):
     c = d.c()
     assert L.ac_conv2d_wgrad_compressed_rect(ctypes.byref(c), 2, 4, 0x10000, 0x10000, 0x10000, 0x10000, 16, None) \
         == ac.api.AC_ERR_WORKSPACE_TOO_SMALL
+
+
+def test_sm_budget_is_a_per_thread_planning_hint(ac):
+    """Fewer SMs to count on: fewer K-slices, fewer CTAs, a smaller workspace; 0 restores the default; another
+    host thread is not affected."""
+    import threading
+    d = ac.ConvDesc(64, 256, 256, 14, 14, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc")
+    assert ac.ac_get_sm_budget() == 148
+    full, full_ws = ac.ac_wgrad_plan_info(d), ac.ac_workspace_bytes(d)
+    try:
+        ac.ac_set_sm_budget(37)
+        assert ac.ac_get_sm_budget() == 37
+        part, part_ws = ac.ac_wgrad_plan_info(d), ac.ac_workspace_bytes(d)
+        assert part["groups"] == full["groups"] and part["ctas"] <= 37 < full["ctas"]
+        assert part["splits"] < full["splits"] and part_ws < full_ws
+        assert part_ws == 256 + part["splits"] * 4 * 256 * 256 * 9
+        seen = []
+        t = threading.Thread(target=lambda: seen.append((ac.ac_get_sm_budget(), ac.ac_workspace_bytes(d))))
+        t.start(); t.join()
+        assert seen == [(148, full_ws)]
+        with pytest.raises(ac.AcError):
+            ac.ac_set_sm_budget(-1)
+        assert ac.ac_get_sm_budget() == 37
+        ac.ac_set_sm_budget(10 ** 6)
+        assert ac.ac_get_sm_budget() == 148
+    finally:
+        ac.ac_set_sm_budget(0)
+    assert ac.ac_workspace_bytes(d) == full_ws

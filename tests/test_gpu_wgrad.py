@@ -510,3 +510,42 @@ def test_stride_above_k_matches_checker(case):
     assert ac.ac_wgrad_plan_info(d)["tensor_core"] in ((code,) if code != 3 else (3, 4))
     err, got, want = wgrad_error_full(d)
     assert err <= TOL_DW[dtype], err
+
+
+def test_sm_budget_layers_side_by_side_match_checker():
+    """Four layers planned for a quarter of the SMs each, enqueued on four streams without synchronising in
+    between: every dW against the checker, and against the same call planned for the whole GPU."""
+    import torch
+    import oracle
+    import paper_2409_11902_b200 as ac
+    from paper_2409_11902_b200 import synth
+    shapes = [(6, 64, 64, 28, 28, 3, 3, 1, 1, 2), (6, 128, 128, 14, 14, 3, 3, 1, 1, 2),
+              (6, 256, 128, 14, 14, 1, 1, 1, 0, 2), (6, 128, 128, 28, 28, 3, 3, 2, 1, 2)]
+    work = []
+    for i, sh in enumerate(shapes):
+        d = D(*sh, "bf16", "nhwc")
+        z, dy = make_wgrad_inputs(d, seed=20 + i)
+        want = oracle.wgrad_compressed(synth.to_f64(z), synth.to_f64(dy), d.H, d.W, d.R, d.S, d.stride, d.pad, d.k)
+        work.append(dict(d=d, z=synth.to_layout(z, "nhwc").cuda(), dy=synth.to_layout(dy, "nhwc").cuda(), want=want,
+                         whole=run_wgrad(d, z, dy)))
+    try:
+        ac.ac_set_sm_budget(37)
+        for w in work:
+            n = ac.ac_workspace_bytes(w["d"])
+            assert ac.ac_wgrad_plan_info(w["d"])["ctas"] <= 37
+            w["ws"] = torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
+            w["dw"] = torch.full(w["d"].dw_shape, float("nan"), device="cuda")
+            w["stream"] = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        for rep in range(3):
+            for w in work:
+                with torch.cuda.stream(w["stream"]):
+                    ac.ac_conv2d_wgrad_compressed(w["d"], w["z"], w["dy"], w["dw"], w["ws"])
+        torch.cuda.synchronize()
+    finally:
+        ac.ac_set_sm_budget(0)
+    for w in work:
+        assert ac.ac_workspace_status(w["ws"])[0] == 0
+        got = w["dw"].double().cpu().numpy().transpose(0, 3, 1, 2)
+        assert_dw_close(got, w["want"], "bf16")
+        assert_dw_close(got, w["whole"], "bf16")
