@@ -533,12 +533,13 @@ def run_ours(args):
 
 def peak_memory_block(args, dev):
     """Peak device memory of one ResNet-50 training step with the conv inputs saved whole, saved
-    compressed, and saved compressed with 1-bit ReLU masks (Section 3's points of interest)."""
+    compressed, and saved compressed with 1-bit ReLU masks (Section 3's points of interest), and the
+    duration of two further steps per scheme (step_ms)."""
     try:
         from paper_2409_11902_b200 import train_step
     except ImportError:
         return None
-    return train_step.peak_memory_report(batch=args.peak_memory_batch, k=K_POOL, device=dev)
+    return train_step.peak_memory_report(batch=args.peak_memory_batch, k=K_POOL, device=dev, time_steps=2)
 
 
 def cpu_baseline(layers, host, n_frac):

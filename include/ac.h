@@ -124,6 +124,25 @@ ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z
                                 void *mask, void *stream);
 
 /*
+ * The backward pass of that ReLU, from the mask alone: dx[i] = dy[i] if bit i of
+ * the mask is set, else 0, for the N*C_in*H*W elements of the tensor in memory
+ * order (the bit order ac_compress_relu_mask writes; the layout does not matter
+ * as long as dy and dx use the one the mask was taken in). This is what lets the
+ * ReLU drop its output: Section 4 removes the convolution's claim on X, this
+ * call the ReLU's.
+ *
+ *   mask  in : ceil(N*C_in*H*W / 8) bytes, as written by ac_compress_relu_mask.
+ *   dy    in : gradient with respect to the ReLU's output, desc->dtype.
+ *   dx    out: gradient with respect to its input, desc->dtype; may alias dy.
+ * N*C_in*H*W must be a multiple of 8 (AC_ERR_UNSUPPORTED otherwise; the mask
+ * kernels have the same domain). All three pointers 16-byte aligned; one kernel
+ * launch on `stream`; no scratch memory. Only N, C_in, H, W and dtype of the
+ * descriptor are read.
+ */
+ac_status ac_relu_mask_backward(const ac_conv_desc *desc, const void *mask, const void *dy,
+                                void *dx, void *stream);
+
+/*
  * Weight gradient from the compressed activation (Section 4: Z is expanded to
  * X's shape and the ordinary weight gradient is taken of that; figure:
  * dL/dW ~ Z (*) dL/dY). With Xt[n,c,h,w] = Z[n,c,h/k,w/k] for 0<=h<H, 0<=w<W

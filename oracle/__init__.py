@@ -113,6 +113,14 @@ def relu(a: np.ndarray) -> np.ndarray:
     return y
 
 
+def relu_backward(a: np.ndarray, dy: np.ndarray) -> np.ndarray:
+    """Gradient of Y = max(A, 0) with respect to A: dY where A > 0, else 0 (the value 0 at A = 0 is
+    the one a sign mask `A > 0` stands for)."""
+    a, dy = _c(a), _c(dy)
+    assert a.shape == dy.shape
+    return np.where(a > 0, dy, 0.0)
+
+
 def wgrad_dense(x, dy, R, S, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
     """Ordinary convolution weight gradient, dW [Co,Ci,R,S]."""
     x, dy = _c(x), _c(dy)

@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.ac_compress.argtypes = [dp, vp, vp, vp, vp]
         L.ac_compress_relu_mask.restype = ctypes.c_int
         L.ac_compress_relu_mask.argtypes = [dp, vp, vp, vp, vp]
+        L.ac_relu_mask_backward.restype = ctypes.c_int
+        L.ac_relu_mask_backward.argtypes = [dp, vp, vp, vp, vp]
         L.ac_conv2d_wgrad_compressed.restype = ctypes.c_int
         L.ac_conv2d_wgrad_compressed.argtypes = [dp, vp, vp, vp, vp, sz, vp]
         L.ac_accumulate_workspace_bytes.restype = sz
@@ -202,6 +204,14 @@ def ac_compress_relu_mask(desc: ConvDesc, a, z, mask, stream=None) -> None:
     st = lib().ac_compress_relu_mask(ctypes.byref(c), _ptr(a), _ptr(z), _ptr(mask), _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_compress_relu_mask")
+
+
+def ac_relu_mask_backward(desc: ConvDesc, mask, dy, dx, stream=None) -> None:
+    """dx = dy where the mask's bit is set, else 0 (elements in memory order); dx may be dy."""
+    c = desc.c()
+    st = lib().ac_relu_mask_backward(ctypes.byref(c), _ptr(mask), _ptr(dy), _ptr(dx), _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_relu_mask_backward")
 
 
 def ac_conv2d_wgrad_compressed(desc: ConvDesc, z, dy, dw, workspace, workspace_bytes=None,

@@ -7,6 +7,8 @@ namespace {
 thread_local int g_sm_budget = kNumSMs;
 }
 
+ac_status launch_relu_mask_backward(const Dims& d, const void* mask, const void* dy, void* dx, cudaStream_t st);   // compress.cu
+
 ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o, int k_h, int k_w) {
     if (!d || !o) return AC_ERR_INVALID_ARG;
     *o = Dims{};   // plans are cached by the bytes of this struct
@@ -174,6 +176,16 @@ ac_status ac_compress_relu_mask(const ac_conv_desc* desc, const void* a, void* z
     if (!a || !z || !mask) return AC_ERR_INVALID_ARG;
     if (!aligned16(a) || !aligned16(z) || !aligned16(mask)) return AC_ERR_MISALIGNED;
     return launch_compress_mask(d, a, z, mask, static_cast<cudaStream_t>(stream));
+}
+
+ac_status ac_relu_mask_backward(const ac_conv_desc* desc, const void* mask, const void* dy, void* dx,
+                                void* stream) {
+    Dims d;
+    ac_status st = make_dims(desc, false, &d);
+    if (st != AC_OK) return st;
+    if (!mask || !dy || !dx) return AC_ERR_INVALID_ARG;
+    if (!aligned16(mask) || !aligned16(dy) || !aligned16(dx)) return AC_ERR_MISALIGNED;
+    return launch_relu_mask_backward(d, mask, dy, dx, static_cast<cudaStream_t>(stream));
 }
 
 ac_status ac_conv2d_wgrad_compressed(const ac_conv_desc* desc, const void* z, const void* dy,

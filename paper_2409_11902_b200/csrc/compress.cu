@@ -512,4 +512,49 @@ ac_status launch_compress_mask(const Dims& d, const void* a, void* z, void* mask
     return launch_typed<B, 2>(d, (const B*)a, (B*)z, nullptr, (unsigned char*)mask, st);
 }
 
+// ReLU backward from the sign mask: dx[i] = bit i of the mask ? dy[i] : 0, eight elements (one mask byte) per thread.
+namespace {
+template <typename T>
+__global__ void __launch_bounds__(256)
+relu_mask_backward_kernel(const unsigned char* __restrict__ mask, const T* dy, T* dx, long long groups) {
+    constexpr int V = 16 / (int)sizeof(T);      // elements per 16-byte vector
+    const long long g = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (g >= groups) return;
+    const unsigned int m = mask[g];
+    const uint4* src = reinterpret_cast<const uint4*>(dy + g * 8);
+    uint4* dst = reinterpret_cast<uint4*>(dx + g * 8);
+#pragma unroll
+    for (int v = 0; v < 8 / V; ++v) {
+        uint4 q = src[v];
+        uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (sizeof(T) == 4) {
+                if (!((m >> (v * 4 + j)) & 1u)) w[j] = 0u;
+            } else {
+                const unsigned int b = m >> (v * 8 + 2 * j);
+                w[j] &= ((b & 1u) ? 0x0000ffffu : 0u) | ((b & 2u) ? 0xffff0000u : 0u);
+            }
+        }
+        dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+}  // namespace
+
+ac_status launch_relu_mask_backward(const Dims& d, const void* mask, const void* dy, void* dx, cudaStream_t st) {
+    const long long n = d.x_elems();
+    if (n % 8 != 0) return AC_ERR_UNSUPPORTED;
+    const long long groups = n / 8, blocks = (groups + 255) / 256;
+    if (blocks >= (1ll << 31)) return AC_ERR_UNSUPPORTED;
+    if (d.dtype == AC_F32)
+        relu_mask_backward_kernel<float><<<(unsigned)blocks, 256, 0, st>>>(
+            static_cast<const unsigned char*>(mask), static_cast<const float*>(dy), static_cast<float*>(dx), groups);
+    else
+        relu_mask_backward_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(
+            static_cast<const unsigned char*>(mask), static_cast<const __nv_bfloat16*>(dy),
+            static_cast<__nv_bfloat16*>(dx), groups);
+    AC_CUDA_TRY(cudaGetLastError());
+    return AC_OK;
+}
+
 }  // namespace ac

@@ -81,7 +81,12 @@ class CompressedConv(torch.autograd.Function):
         dx = None
         if ctx.needs_input_grad[0]:
             w = w_master.to(torch.bfloat16).contiguous(memory_format=torch.channels_last)
-            dx = torch.nn.grad.conv2d_input(ctx.x_shape, w, dy, ctx.stride, ctx.pad)
+            # the input gradient is the transposed convolution of dY (the framework's own kernel for it; the
+            # generic conv2d_input helper would first materialise a dummy input of X's size)
+            H, W = ctx.x_shape[2], ctx.x_shape[3]
+            R, S = w.shape[2], w.shape[3]
+            op = (H - ((dy.shape[2] - 1) * ctx.stride - 2 * ctx.pad + R), W - ((dy.shape[3] - 1) * ctx.stride - 2 * ctx.pad + S))
+            dx = F.conv_transpose2d(dy, w, None, ctx.stride, ctx.pad, op)
         dw = torch.empty((d.C_out, d.R, d.S, d.C_in), dtype=torch.float32, device=dy.device)
         ws = torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dy.device)
         api.ac_conv2d_wgrad_compressed(d, ctx.z, dy, dw, ws)
@@ -112,12 +117,11 @@ class ReluKeepingMask(torch.autograd.Function):
     def backward(ctx, dy):
         dy = _nhwc(dy)
         N, C, H, W = dy.shape
-        # bit i of the mask = element i in channels-last memory order, least significant bit first
-        shifts = torch.arange(8, device=dy.device, dtype=torch.uint8)
-        bits = ((ctx.mask.unsqueeze(1) >> shifts) & 1).reshape(-1)[:dy.numel()]
-        keep = bits.view(N, H, W, C).permute(0, 3, 1, 2).to(dy.dtype)
+        d = api.ConvDesc(N, C, C, H, W, 1, 1, (1, 1), (0, 0), 1, "bf16", "nhwc")
+        dx = torch.empty_like(dy)      # channels-last, like dy
+        api.ac_relu_mask_backward(d, ctx.mask, dy, dx)
         ctx.mask = None
-        return dy * keep, None, None
+        return dx, None, None
 
 
 class ResNet50:
@@ -203,7 +207,7 @@ def synthetic_batch(batch, device, seed=0, num_classes=1000):
     return images.to(device).contiguous(memory_format=torch.channels_last), labels.to(device)
 
 
-def training_step(scheme, batch=256, k=2, device="cuda", seed=0, compress_stem=True, capture=None):
+def training_step(scheme, batch=256, k=2, device="cuda", seed=0, compress_stem=True, capture=None, time_steps=0):
     """Runs one step and reads the allocator at Section 3's five points. Returns a dict with the
     loss and the bytes; `capture`: a list that receives (desc, X, Z, dY, dW) of every compressed
     convolution's backward (for checks; X is then copied in the forward pass, so the memory figures of such
@@ -239,14 +243,30 @@ def training_step(scheme, batch=256, k=2, device="cuda", seed=0, compress_stem=T
     out["mib"]["step_peak"] = max(out["mib"]["3_forward_peak"], out["mib"]["backward_peak"],
                                   out["mib"]["5_optimizer_peak"])
     out["grad_norm"] = float(torch.sqrt(sum((p.grad.double() ** 2).sum() for p in model.params if p.grad is not None)))
+    if time_steps > 0 and capture is None:
+        # duration of further whole steps (forward, backward, optimizer), CUDA events on the current stream
+        del logits, loss
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(time_steps):
+            opt.zero_grad(set_to_none=True)
+            lg = model.forward(images)
+            ls = F.cross_entropy(lg.float(), labels)
+            ls.backward()
+            opt.step()
+            del lg, ls
+        e1.record()
+        torch.cuda.synchronize(dev)
+        out["step_ms"] = e0.elapsed_time(e1) / time_steps
+        logits = loss = None
     del model, opt, images, labels, logits, loss
     torch.cuda.empty_cache()
     return out
 
 
-def peak_memory_report(batch=256, k=2, device="cuda", compress_stem=True):
+def peak_memory_report(batch=256, k=2, device="cuda", compress_stem=True, time_steps=0):
     """The step under each scheme, and the reduction of the peak against scheme "full"."""
-    runs = {s: training_step(s, batch, k, device, compress_stem=compress_stem) for s in SCHEMES}
+    runs = {s: training_step(s, batch, k, device, compress_stem=compress_stem, time_steps=time_steps) for s in SCHEMES}
     full = runs["full"]["mib"]
     rep = {"model": "ResNet-50 (53 convolutions), bf16 channels-last, fp32 master weights, SGD momentum",
            "batch": batch, "k": k, "compress_stem": compress_stem,
@@ -269,5 +289,6 @@ if __name__ == "__main__":
     ap.add_argument("--batch", type=int, default=256)
     ap.add_argument("--k", type=int, default=2)
     ap.add_argument("--no-stem", action="store_true", help="leave the first convolution uncompressed")
+    ap.add_argument("--time-steps", type=int, default=0, help="also time this many further steps per scheme (step_ms)")
     a = ap.parse_args()
-    print(json.dumps(peak_memory_report(a.batch, a.k, "cuda:0", not a.no_stem), indent=1))
+    print(json.dumps(peak_memory_report(a.batch, a.k, "cuda:0", not a.no_stem, a.time_steps), indent=1))

@@ -83,6 +83,50 @@ def test_fused_relu_compress_sign_mask(shape, k, dtype, layout):
         assert e.value.status == ac.api.AC_ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(3, 64, 56, 56), (2, 512, 7, 7), (2, 32, 16, 64), (1, 8, 3, 5), (5, 8, 3, 40)])
+def test_relu_backward_from_the_sign_mask(shape, dtype, layout):
+    """ac_relu_mask_backward on the mask ac_compress_relu_mask wrote: bit for bit dY where A > 0, else 0 -- into a
+    buffer of its own and in place."""
+    import numpy as np
+    import torch
+    import oracle
+    import paper_2409_11902_b200 as ac
+    from helpers import canary_intact, padded_empty
+    from paper_2409_11902_b200 import synth
+    d = desc(*shape, 1, dtype, layout)
+    a = synth.pre_activation(3, shape, dtype)
+    dy = synth.grad_output(3, shape, dtype)
+    n_el = int(np.prod(shape))
+    ad, dyd = synth.to_layout(a, layout).cuda(), synth.to_layout(dy, layout).cuda()
+    z = torch.empty(d.z_shape, dtype=d.torch_dtype, device="cuda")
+    mask = torch.empty((n_el + 7) // 8, dtype=torch.uint8, device="cuda")
+    ac.ac_compress_relu_mask(d, ad, z, mask)
+    want = oracle.relu_backward(synth.to_f64(a), synth.to_f64(dy))
+    xbuf, dx, xspan = padded_empty(tuple(dyd.shape), d.torch_dtype, "cuda:0")
+    dx.fill_(float("nan"))
+    keep = dyd.clone()
+    ac.ac_relu_mask_backward(d, mask, dyd, dx)
+    torch.cuda.synchronize()
+    assert canary_intact(xbuf, xspan) and torch.equal(dyd.view(torch.uint8), keep.view(torch.uint8))
+    assert np.array_equal(synth.to_f64(synth.from_layout(dx.cpu(), layout)), want)
+    ac.ac_relu_mask_backward(d, mask, dyd, dyd)      # in place
+    torch.cuda.synchronize()
+    assert np.array_equal(synth.to_f64(synth.from_layout(dyd.cpu(), layout)), want)
+
+
+def test_relu_mask_backward_rejects_what_it_cannot_take():
+    import torch
+    import paper_2409_11902_b200 as ac
+    d = desc(1, 3, 5, 5, 1, "bf16", "nhwc")      # 75 elements: not a multiple of 8
+    t = torch.zeros(128, dtype=torch.bfloat16, device="cuda")
+    m = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(ac.AcError) as e:
+        ac.ac_relu_mask_backward(d, m, t, t)
+    assert e.value.status == ac.api.AC_ERR_UNSUPPORTED
+
+
 def test_large_map_many_blocks():
     # 64 x 128 x 64 x 64 fp32 = 128 MiB: larger than L2, > 100k thread blocks
     for layout in ("nchw", "nhwc"):

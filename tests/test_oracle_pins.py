@@ -126,6 +126,26 @@ def test_relu():
     assert np.array_equal(oracle.relu(a), np.maximum(a, 0.0))
 
 
+def test_relu_backward_is_the_derivative_of_relu():
+    """Central differences of L = sum(relu(A) * dY) in A (exact away from 0: L is piecewise linear), the value 0
+    at A = 0, and equality with the sign mask applied to dY."""
+    a = RNG.standard_normal(200)
+    a[::17] = 0.0
+    dy = RNG.standard_normal(200)
+    got = oracle.relu_backward(a, dy)
+    h = 1e-3
+    away = np.abs(a) > 2 * h
+    for i in np.flatnonzero(away)[:60]:
+        ap, am = a.copy(), a.copy()
+        ap[i] += h
+        am[i] -= h
+        fd = (np.sum(oracle.relu(ap) * dy) - np.sum(oracle.relu(am) * dy)) / (2 * h)
+        assert abs(fd - got[i]) <= 1e-9 * max(1.0, abs(dy[i]))
+    assert not got[a == 0].any() and not got[a < 0].any()
+    bits = np.unpackbits(np.packbits(a > 0, bitorder="little"), bitorder="little")[:a.size].astype(bool)
+    assert np.array_equal(got, np.where(bits, dy, 0.0))
+
+
 # ---------------------------------------------------------------------- wgrad
 
 CONV_CASES = [
