@@ -124,6 +124,16 @@ ac_status ac_compress_relu_mask(const ac_conv_desc *desc, const void *a, void *z
                                 void *mask, void *stream);
 
 /*
+ * The same pass for a caller that does need Y = max(A, 0) afterwards (as the
+ * input of the next convolution's forward pass) but not for the ReLU's
+ * backward: writes Y as ac_compress with y_out does, Z, and the mask, reading A
+ * once. y_out may alias a (the ReLU in place). Same domain, alignment and
+ * errors as ac_compress_relu_mask; y_out must not be NULL.
+ */
+ac_status ac_compress_relu_mask_y(const ac_conv_desc *desc, const void *a, void *y_out, void *z,
+                                  void *mask, void *stream);
+
+/*
  * The backward pass of that ReLU, from the mask alone: dx[i] = dy[i] if bit i of
  * the mask is set, else 0, for the N*C_in*H*W elements of the tensor in memory
  * order (the bit order ac_compress_relu_mask writes; the layout does not matter

@@ -5,7 +5,7 @@
 """
 from . import synth  # noqa: F401
 from .api import (  # noqa: F401
-    AcError, ConvDesc, ac_backward_step_host, ac_compress, ac_compress_relu_mask, ac_relu_mask_backward, ac_accumulate_workspace_bytes,
+    AcError, ConvDesc, ac_backward_step_host, ac_compress, ac_compress_relu_mask, ac_compress_relu_mask_y, ac_relu_mask_backward, ac_accumulate_workspace_bytes,
     ac_conv2d_wgrad_compressed_accumulate,
     ac_conv2d_wgrad_compressed,
     ac_conv2d_wgrad_compressed_static, ac_collapsed_workspace_bytes,

@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.ac_compress.argtypes = [dp, vp, vp, vp, vp]
         L.ac_compress_relu_mask.restype = ctypes.c_int
         L.ac_compress_relu_mask.argtypes = [dp, vp, vp, vp, vp]
+        L.ac_compress_relu_mask_y.restype = ctypes.c_int
+        L.ac_compress_relu_mask_y.argtypes = [dp, vp, vp, vp, vp, vp]
         L.ac_relu_mask_backward.restype = ctypes.c_int
         L.ac_relu_mask_backward.argtypes = [dp, vp, vp, vp, vp]
         L.ac_conv2d_wgrad_compressed.restype = ctypes.c_int
@@ -204,6 +206,14 @@ def ac_compress_relu_mask(desc: ConvDesc, a, z, mask, stream=None) -> None:
     st = lib().ac_compress_relu_mask(ctypes.byref(c), _ptr(a), _ptr(z), _ptr(mask), _stream(stream))
     if st != AC_OK:
         raise AcError(st, "ac_compress_relu_mask")
+
+
+def ac_compress_relu_mask_y(desc: ConvDesc, a, y_out, z, mask, stream=None) -> None:
+    """Y = max(A, 0) (y_out may be a), Z = pool(Y) and the sign mask in one pass."""
+    c = desc.c()
+    st = lib().ac_compress_relu_mask_y(ctypes.byref(c), _ptr(a), _ptr(y_out), _ptr(z), _ptr(mask), _stream(stream))
+    if st != AC_OK:
+        raise AcError(st, "ac_compress_relu_mask_y")
 
 
 def ac_relu_mask_backward(desc: ConvDesc, mask, dy, dx, stream=None) -> None:

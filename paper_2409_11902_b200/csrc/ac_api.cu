@@ -8,6 +8,7 @@ thread_local int g_sm_budget = kNumSMs;
 }
 
 ac_status launch_relu_mask_backward(const Dims& d, const void* mask, const void* dy, void* dx, cudaStream_t st);   // compress.cu
+ac_status launch_compress_mask_y(const Dims& d, const void* a, void* y, void* z, void* mask, cudaStream_t st);      // compress.cu
 
 ac_status make_dims(const ac_conv_desc* d, bool need_conv, Dims* o, int k_h, int k_w) {
     if (!d || !o) return AC_ERR_INVALID_ARG;
@@ -176,6 +177,16 @@ ac_status ac_compress_relu_mask(const ac_conv_desc* desc, const void* a, void* z
     if (!a || !z || !mask) return AC_ERR_INVALID_ARG;
     if (!aligned16(a) || !aligned16(z) || !aligned16(mask)) return AC_ERR_MISALIGNED;
     return launch_compress_mask(d, a, z, mask, static_cast<cudaStream_t>(stream));
+}
+
+ac_status ac_compress_relu_mask_y(const ac_conv_desc* desc, const void* a, void* y_out, void* z, void* mask,
+                                  void* stream) {
+    Dims d;
+    ac_status st = make_dims(desc, false, &d);
+    if (st != AC_OK) return st;
+    if (!a || !y_out || !z || !mask) return AC_ERR_INVALID_ARG;
+    if (!aligned16(a) || !aligned16(y_out) || !aligned16(z) || !aligned16(mask)) return AC_ERR_MISALIGNED;
+    return launch_compress_mask_y(d, a, y_out, z, mask, static_cast<cudaStream_t>(stream));
 }
 
 ac_status ac_relu_mask_backward(const ac_conv_desc* desc, const void* mask, const void* dy, void* dx,

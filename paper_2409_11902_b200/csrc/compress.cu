@@ -127,16 +127,16 @@ __device__ __forceinline__ void store_mask(unsigned char* mask, long long elem_o
 // time, all loads of up to four rows issued before the first use; K = 0: any k.
 // x is not __restrict__: the fused ReLU may run in place (y == x); a thread reads its own
 // elements before it writes them and no other thread touches them.
-template <typename T, int K, int MODE>   // MODE 0: pool only, 1: also store max(x,0), 2: also store the sign mask
+template <typename T, int K, int MODE>   // MODE 0: pool only, 1: also store max(x,0), 2: also store the sign mask, 3: both
 __global__ void __launch_bounds__(256)
 compress_nhwc_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int CV,
                   int kh, int kw, int Hp, int Wp) {
     pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
-    constexpr bool RELU = MODE != 0;
+    constexpr bool RELU = MODE != 0, STORE_Y = MODE == 1 || MODE == 3, MASK = MODE >= 2;
     constexpr int VW = VecTraits<T>::VW;
     const unsigned item = blockIdx.x * 256u + threadIdx.x;
     const bool in_range = item < (unsigned)Wp * (unsigned)CV;
-    const unsigned lanes = MODE == 2 ? __ballot_sync(0xffffffffu, in_range) : 0u;   // pairs leave together
+    const unsigned lanes = MASK ? __ballot_sync(0xffffffffu, in_range) : 0u;   // pairs leave together
     if (!in_range) return;
     const int q = (int)(item / (unsigned)CV);
     const int cv = (int)(item - (unsigned)q * (unsigned)CV);
@@ -160,7 +160,7 @@ compress_nhwc_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int 
                     const int h = h0 + hb + dh, w = w0 + dw;
                     raw[dh][dw] = make_uint4(0, 0, 0, 0);
                     if (h < h1 && w < w1)
-                        raw[dh][dw] = load16<MODE != 1>(x + ((((n * H + h) * (long long)W + w) * CV + cv) * VW));
+                        raw[dh][dw] = load16<!STORE_Y>(x + ((((n * H + h) * (long long)W + w) * CV + cv) * VW));
                 }
 #pragma unroll
             for (int dh = 0; dh < KR; ++dh) {
@@ -172,10 +172,10 @@ compress_nhwc_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int 
                     const int h = h0 + hb + dh, w = w0 + dw;
                     float f[VW];
                     unpack<T, RELU>(raw[dh][dw], f);
-                    if (MODE == 1 && h < h1 && w < w1)
+                    if (STORE_Y && h < h1 && w < w1)
                         *reinterpret_cast<uint4*>(y + ((((n * H + h) * (long long)W + w) * CV + cv) * VW)) =
                             raw[dh][dw];
-                    if (MODE == 2)
+                    if (MASK)
                         store_mask<VW>(mask, (((n * H + h) * (long long)W + w) * CV + cv) * VW,
                                        positive_bits<T>(raw[dh][dw], f), h < h1 && w < w1, lanes);
 #pragma unroll
@@ -193,10 +193,10 @@ compress_nhwc_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int 
             const long long rbase = ((n * H + h) * (long long)W) * CV + cv;
             for (int w = w0; w < w1; ++w) {
                 const long long off = (rbase + (long long)w * CV) * VW;
-                uint4 raw = load16<MODE != 1>(x + off);
+                uint4 raw = load16<!STORE_Y>(x + off);
                 float f[VW];
                 unpack<T, RELU>(raw, f);
-                if (MODE == 1) *reinterpret_cast<uint4*>(y + off) = raw;
+                if (STORE_Y) *reinterpret_cast<uint4*>(y + off) = raw;
 #pragma unroll
                 for (int i = 0; i < VW; ++i) row[i] += f[i];
             }
@@ -222,7 +222,7 @@ ac_status launch_nhwc_vec(const T* x, T* z, T* y, unsigned char* mask, long long
         case 4: compress_nhwc_vec<T, 4, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, kh, kw, Hp, Wp); break;
         case 8: compress_nhwc_vec<T, 8, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, kh, kw, Hp, Wp); break;
         default:
-            if (MODE == 2) return AC_ERR_UNSUPPORTED;   // the mask needs warp-uniform loops
+            if (MODE >= 2) return AC_ERR_UNSUPPORTED;   // the mask needs warp-uniform loops
             compress_nhwc_vec<T, 0, MODE><<<grid, 256, 0, st>>>(x, z, y, mask, H, W, CV, kh, kw, Hp, Wp);
             break;
     }
@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(256)
 compress_nchw_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int H, int W, int Hp,
                   int Wp, long long total) {
     pdl_launch_dependents();   // a weight-gradient kernel queued behind this one may begin its set-up
-    constexpr bool RELU = MODE != 0;
+    constexpr bool RELU = MODE != 0, STORE_Y = MODE == 1 || MODE == 3, MASK = MODE >= 2;
     constexpr int VW = VecTraits<T>::VW;
     const int WV = W / VW;
     I idx = (I)blockIdx.x * 256u + threadIdx.x;     // I = unsigned when the item count fits 32 bits
@@ -262,15 +262,15 @@ compress_nchw_vec(const T* x, T* __restrict__ z, T* y, unsigned char* mask, int 
         const long long off = ((nc * H + h) * (long long)WV + wv) * VW;
         unsigned bits = 0;
         if (h < h1) {
-            uint4 raw = load16<MODE != 1>(x + off);
+            uint4 raw = load16<!STORE_Y>(x + off);
             float f[VW];
             unpack<T, RELU>(raw, f);
-            if (MODE == 1 && active) *reinterpret_cast<uint4*>(y + off) = raw;
-            if (MODE == 2) bits = positive_bits<T>(raw, f);
+            if (STORE_Y && active) *reinterpret_cast<uint4*>(y + off) = raw;
+            if (MASK) bits = positive_bits<T>(raw, f);
 #pragma unroll
             for (int i = 0; i < VW; ++i) acc[i] += f[i];
         }
-        if (MODE == 2) store_mask<VW>(mask, off, bits, active && h < h1, 0xffffffffu);
+        if (MASK) store_mask<VW>(mask, off, bits, active && h < h1, 0xffffffffu);
     }
     const float inv = 1.0f / (float)((h1 - h0) * K);
     if (K <= VW) {
@@ -436,7 +436,7 @@ void launch_nchw_vec(const Dims& d, const T* x, T* z, T* y, unsigned char* mask,
                                                                               d.Wp, total);
 }
 
-// MODE 2 (sign mask) runs on the vector kernels only: a mask byte covers 8 consecutive elements,
+// MODE 2 and 3 (sign mask) run on the vector kernels only: a mask byte covers 8 consecutive elements,
 // so C (NHWC) or W (NCHW) must be a multiple of 8 and k one of 1, 2, 4, 8.
 template <typename T, int MODE>
 ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, unsigned char* mask, cudaStream_t st) {
@@ -445,25 +445,25 @@ ac_status launch_typed(const Dims& d, const T* x, T* z, T* y, unsigned char* mas
     if (zt >= (1ll << 31) * 256) return AC_ERR_UNSUPPORTED;
     const bool square = d.kh == d.kw;
     const bool pow2k = square && (d.k == 2 || d.k == 4 || d.k == 8);
-    if (square && d.k == 1 && d.x_elems() % (MODE == 2 ? 8 : VW) == 0) {
+    if (square && d.k == 1 && d.x_elems() % (MODE >= 2 ? 8 : VW) == 0) {
         // a copy (or a plain ReLU): treat the tensor as one row of 16-byte vectors
         const long long nv = d.x_elems() / VW;
         if (nv < (1ll << 31))
             return launch_nhwc_vec<T, MODE>(x, z, y, mask, 1, 1, (int)nv, 1, 1, 1, 1, (int)nv, st);
     }
-    if (d.layout == AC_NHWC && d.Ci % (MODE == 2 ? 8 : VW) == 0) {
+    if (d.layout == AC_NHWC && d.Ci % (MODE >= 2 ? 8 : VW) == 0) {
         const ac_status st_ =
             launch_nhwc_vec<T, MODE>(x, z, y, mask, d.N, d.H, d.W, d.Ci / VW, d.kh, d.kw, d.Hp, d.Wp, st);
         if (st_ != AC_ERR_UNSUPPORTED) return st_;
     }
-    if (d.layout == AC_NCHW && pow2k && d.W % (MODE == 2 ? 8 : VW) == 0 && d.W % d.k == 0 &&
+    if (d.layout == AC_NCHW && pow2k && d.W % (MODE >= 2 ? 8 : VW) == 0 && d.W % d.k == 0 &&
         (VW % d.k == 0 || d.k == 2 * VW)) {
         const long long total = (long long)d.N * d.Ci * d.Hp * (d.W / VW);
         if (d.k == 2) launch_nchw_vec<T, 2, MODE>(d, x, z, y, mask, total, st);
         else if (d.k == 4) launch_nchw_vec<T, 4, MODE>(d, x, z, y, mask, total, st);
         else launch_nchw_vec<T, 8, MODE>(d, x, z, y, mask, total, st);
     } else {
-        if (MODE == 2) return AC_ERR_UNSUPPORTED;
+        if (MODE >= 2) return AC_ERR_UNSUPPORTED;
         if (const int rb = rows_per_block<T>(d)) {
             const long long out_el = (long long)d.Wp * d.Ci;
             const int vec_out = (out_el % VW == 0) ? 1 : 0;     // then every pooled row starts 16-byte aligned
@@ -510,6 +510,15 @@ ac_status launch_compress_mask(const Dims& d, const void* a, void* z, void* mask
         return launch_typed<float, 2>(d, (const float*)a, (float*)z, nullptr, (unsigned char*)mask, st);
     using B = __nv_bfloat16;
     return launch_typed<B, 2>(d, (const B*)a, (B*)z, nullptr, (unsigned char*)mask, st);
+}
+
+// the same, also storing Y = max(A, 0) (y may be a)
+ac_status launch_compress_mask_y(const Dims& d, const void* a, void* y, void* z, void* mask, cudaStream_t st) {
+    if (d.x_elems() % 8 != 0) return AC_ERR_UNSUPPORTED;
+    if (d.dtype == AC_F32)
+        return launch_typed<float, 3>(d, (const float*)a, (float*)z, (float*)y, (unsigned char*)mask, st);
+    using B = __nv_bfloat16;
+    return launch_typed<B, 3>(d, (const B*)a, (B*)z, (B*)y, (unsigned char*)mask, st);
 }
 
 // ReLU backward from the sign mask: dx[i] = bit i of the mask ? dy[i] : 0, eight elements (one mask byte) per thread.

@@ -98,7 +98,7 @@ class CompressedConv(torch.autograd.Function):
 
 class ReluKeepingMask(torch.autograd.Function):
     """y = max(a, 0) in place. Keeps one bit per element, and leaves Z = pool_k(y) in `saved`
-    for the convolutions that read y."""
+    for the convolutions that read y (`ac_compress_relu_mask_y`); backward: `ac_relu_mask_backward`."""
 
     @staticmethod
     def forward(ctx, a, saved, k):
@@ -108,10 +108,10 @@ class ReluKeepingMask(torch.autograd.Function):
         saved.z = torch.empty((N, C, d.Hp, d.Wp), dtype=torch.bfloat16, device=a.device,
                               memory_format=torch.channels_last)
         mask = torch.empty((a.numel() + 7) // 8, dtype=torch.uint8, device=a.device)
-        api.ac_compress_relu_mask(d, a, saved.z, mask)
+        api.ac_compress_relu_mask_y(d, a, a, saved.z, mask)      # the ReLU in place, Z and the mask: one pass over A
         ctx.mask = mask
         ctx.mark_dirty(a)
-        return a.relu_()
+        return a
 
     @staticmethod
     def backward(ctx, dy):

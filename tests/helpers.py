@@ -124,9 +124,10 @@ def run_compress(d: ac.ConvDesc, seed=0, fused_relu=False, inplace=False, dev="c
     return compress_error(z64, x64, d.k), z64, x64
 
 
-def run_compress_mask(d: ac.ConvDesc, seed=0, dev="cuda:0"):
+def run_compress_mask(d: ac.ConvDesc, seed=0, dev="cuda:0", store_y=None):
     """The mask form of the fused call. Returns the pooling error; the mask is compared bit for
-    bit with (A > 0) in memory order."""
+    bit with (A > 0) in memory order. `store_y`: "own" or "inplace" runs the variant that also writes
+    Y = max(A, 0), into a buffer of its own or over A."""
     shape = (d.N, d.C_in, d.H, d.W)
     a = synth.pre_activation(seed, shape, d.dtype)
     x64 = oracle.relu(synth.to_f64(a))
@@ -135,11 +136,22 @@ def run_compress_mask(d: ac.ConvDesc, seed=0, dev="cuda:0"):
     zbuf, z, zspan = padded_empty(d.z_shape, d.torch_dtype, dev)
     mbuf, m, mspan = padded_empty(((n_el + 7) // 8,), torch.uint8, dev)
     before = ad.clone()
-    ac.ac_compress_relu_mask(d, ad, z, m)
+    if store_y is None:
+        ac.ac_compress_relu_mask(d, ad, z, m)
+    else:
+        ybuf, y, yspan = padded_empty(tuple(ad.shape), d.torch_dtype, dev)
+        y.fill_(float("nan"))
+        out = ad if store_y == "inplace" else y
+        ac.ac_compress_relu_mask_y(d, ad, out, z, m)
+        torch.cuda.synchronize()
+        assert canary_intact(ybuf, yspan), "wrote outside Y"
+        y64 = synth.to_f64(synth.from_layout(out.cpu(), d.layout))
+        assert np.array_equal(y64, x64), "fused ReLU output differs from max(A, 0)"
     torch.cuda.synchronize()
     assert canary_intact(zbuf, zspan), "wrote outside Z"
     assert canary_intact(mbuf, mspan), "wrote outside the mask"
-    assert torch.equal(ad.view(torch.uint8), before.view(torch.uint8)), "the input must not be modified"
+    if store_y != "inplace":
+        assert torch.equal(ad.view(torch.uint8), before.view(torch.uint8)), "the input must not be modified"
     a_mem = synth.to_f64(synth.to_layout(a, d.layout)).reshape(-1)   # memory order of the layout
     want = np.packbits(a_mem > 0, bitorder="little")
     assert np.array_equal(m.cpu().numpy(), want), "sign mask differs from (A > 0)"

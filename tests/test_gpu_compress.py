@@ -75,8 +75,9 @@ def test_fused_relu_compress_sign_mask(shape, k, dtype, layout):
     import paper_2409_11902_b200 as ac
     d = desc(*shape, k, dtype, layout)
     if k != 3 and mask_form_exists(shape, k, layout):
-        err = run_compress_mask(d)
-        assert err <= TOL_Z[dtype], err
+        for store_y in (None, "own", "inplace"):
+            err = run_compress_mask(d, store_y=store_y)
+            assert err <= TOL_Z[dtype], (store_y, err)
     else:
         with pytest.raises(ac.AcError) as e:
             run_compress_mask(d)
