@@ -40,6 +40,9 @@ def main():
     ap.add_argument("--layout", default="nhwc")
     ap.add_argument("--relu", action="store_true", help="use the fused ReLU+compress form")
     ap.add_argument("--mask", action="store_true", help="use the fused ReLU+compress form that keeps a sign mask")
+    ap.add_argument("--relu-ops", action="store_true",
+                    help="instead: the masked ReLU's two passes on the layer's input tensor, forward (ReLU in place + "
+                         "compress + mask, ac_compress_relu_mask_y) and backward (ac_relu_mask_backward)")
     ap.add_argument("--collapsed", action="store_true", help="time the collapsed weight-gradient entry point too")
     a = ap.parse_args()
     ci, co, H, W, R, S, st, pd = LAYERS[a.layer]
@@ -50,6 +53,27 @@ def main():
     z = torch.empty(d.z_shape, dtype=d.torch_dtype, device=dev)
     y = torch.empty_like(x) if a.relu else None
     mask = torch.empty((x.numel() + 7) // 8, dtype=torch.uint8, device=dev) if a.mask else None
+    if a.relu_ops:
+        acts = [synth.to_layout(synth.pre_activation(i, (d.N, ci, H, W), a.dtype), a.layout).to(dev) for i in range(2)]
+        gy = synth.to_layout(synth.grad_output(1, (d.N, ci, H, W), a.dtype), a.layout).to(dev)
+        gx = torch.empty_like(gy)
+        m = torch.empty((x.numel() + 7) // 8, dtype=torch.uint8, device=dev)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        nbytes = x.numel() * x.element_size()
+        for it in range(a.iters):
+            act = acts[it % 2].clone()
+            e[0].record()
+            api.ac_compress_relu_mask_y(d, act, act, z, m)
+            e[1].record()
+            api.ac_relu_mask_backward(d, m, gy, gx)
+            e[2].record()
+            torch.cuda.synchronize()
+            t_f, t_b = e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])
+            fb = 2 * nbytes + z.numel() * z.element_size() + m.numel()
+            bb = 2 * nbytes + m.numel()
+            print(f"iter {it}: relu+compress+mask {t_f * 1e3:.1f} us ({fb / t_f / 1e6:.0f} GB/s), "
+                  f"relu backward from the mask {t_b * 1e3:.1f} us ({bb / t_b / 1e6:.0f} GB/s)")
+        return
     dw = torch.empty(d.dw_shape, dtype=torch.float32, device=dev)
     ws = torch.empty(max(api.ac_workspace_bytes(d), 256), dtype=torch.uint8, device=dev)
     print("plan:", api.ac_wgrad_plan_info(d))
