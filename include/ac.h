@@ -366,7 +366,10 @@ typedef struct {
                                 and W, at most 128 columns, rows of Z a multiple of 16 bytes long): the matrix
                                 is never written to memory; sixteen warps of the kernel build each K-tile
                                 of it in shared memory from a strip of Z rows fetched by TMA, beside the
-                                warp that issues the MMAs (band_rows = whole output rows per K-tile),
+                                warp that issues the MMAs (band_rows = whole output rows per K-tile); a pooling block
+                                that is a multiple k = f * s of the stride s is first re-blocked to k' = s
+                                in the workspace, Z'[p][q] = Z[p/f][q/f] (|X| / s^2 elements: the same
+                                inflated map), and runs as that,
                                 5: bf16 NHWC with fewer than 64 input channels (a 3-channel stem): the
                                 inflated, zero-padded values every output position reads are gathered
                                 into a [positions][taps x C_in] matrix in the workspace (one column

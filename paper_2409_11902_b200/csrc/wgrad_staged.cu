@@ -623,13 +623,66 @@ ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z,
     return AC_OK;
 }
 
-bool gather_supported(const Dims& d) { return gather_fused_supported(d) || gather_geom(d).ok; }
+// Few input channels with a pooling block that is a multiple of the stride (k = 4 or 8 at stride 2): the in-kernel
+// form wants the stride to be a multiple of k. Z re-blocked to k' = stride, Z'[p][q] = Z[p*k'/k][q*k'/k] (the same
+// inflated map: X~[h] = Z[h/k] = Z'[h/k'] when k' divides k), is a tensor of |X| / k'^2 elements that it does take.
+bool reblocked_dims(const Dims& d, Dims* out) {
+    if (gather_fused_supported(d)) return false;
+    if (d.dtype != AC_BF16 || d.layout != AC_NHWC || d.kh != d.kw || d.sh != d.sw) return false;
+    const int k2 = d.sh;
+    if (k2 < 2 || k2 >= d.k || d.k % k2 != 0) return false;
+    Dims r = d;
+    r.k = r.kh = r.kw = k2;
+    r.Hp = (d.H + k2 - 1) / k2;
+    r.Wp = (d.W + k2 - 1) / k2;
+    if (r.z_elems() >= (1ll << 40) || (r.z_elems() + 255) / 256 >= (1ll << 31)) return false;
+    if (!gather_fused_supported(r) || ((long long)r.Wp * r.Ci) % 8 != 0) return false;
+    *out = r;
+    return true;
+}
+
+// eight consecutive elements of a row of Z' (a row is Wp2 * C elements, a multiple of eight: the in-kernel form asks
+// for rows of whole 16-byte units) per thread: eight 2-byte reads of Z, one 16-byte store
+__global__ void __launch_bounds__(256)
+reblock_nhwc_kernel(const unsigned short* __restrict__ z, uint4* __restrict__ z2, int C, int Hp, int Wp,
+                    int Hp2, int Wp2, int f, long long total8) {
+    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (i >= total8) return;
+    const int row8 = Wp2 * C / 8;
+    const int e0 = (int)(i % row8) * 8;
+    long long r = i / row8;
+    const int p = (int)(r % Hp2);
+    const long long n = r / Hp2;
+    const unsigned short* src = z + ((n * Hp + p / f) * (long long)Wp) * C;
+    unsigned short v[8];
+    int q = e0 / C, c = e0 - q * C;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        v[j] = __ldg(src + (q / f) * C + c);
+        if (++c == C) { c = 0; ++q; }
+    }
+    z2[i] = make_uint4(v[0] | (uint32_t)v[1] << 16, v[2] | (uint32_t)v[3] << 16, v[4] | (uint32_t)v[5] << 16,
+                       v[6] | (uint32_t)v[7] << 16);
+}
+
+bool gather_supported(const Dims& d) {
+    Dims r;
+    return gather_fused_supported(d) || reblocked_dims(d, &r) || gather_geom(d).ok;
+}
 
 void plan_gather(const Dims& d, WgradPlan* pl) {
     if (gather_fused_supported(d)) {      // the matrix is built inside the kernel: no staged copy
         *pl = WgradPlan{};
         pl->path = PATH_GATHER;
         pl->bytes = gather_fused_workspace_bytes(d);
+        return;
+    }
+    Dims r;
+    if (reblocked_dims(d, &r)) {          // the re-blocked Z behind the in-kernel form's own workspace
+        *pl = WgradPlan{};
+        pl->path = PATH_GATHER;
+        pl->st_off_z = up256(gather_fused_workspace_bytes(r));
+        pl->bytes = pl->st_off_z + up256((size_t)r.z_elems() * 2);
         return;
     }
     const GatherGeom g = gather_geom(d);
@@ -647,6 +700,11 @@ void gather_plan_info(const Dims& d, ac_plan_info* info) {
         gather_fused_plan_info(d, info);
         return;
     }
+    Dims r;
+    if (reblocked_dims(d, &r)) {
+        gather_fused_plan_info(r, info);
+        return;
+    }
     const GatherGeom g = gather_geom(d);
     tc2_plan_info(g.in, info);
     info->tensor_core = 5;
@@ -655,6 +713,15 @@ void gather_plan_info(const Dims& d, ac_plan_info* info) {
 ac_status launch_wgrad_gather(const Dims& d, const WgradPlan& pl, const void* z, const void* dy, float* dw,
                               void* workspace, cudaStream_t stream) {
     if (gather_fused_supported(d)) return launch_wgrad_gather_fused(d, z, dy, dw, workspace, stream);
+    Dims r;
+    if (reblocked_dims(d, &r)) {
+        uint4* z2 = reinterpret_cast<uint4*>(static_cast<char*>(workspace) + pl.st_off_z);
+        const long long total8 = r.z_elems() / 8;
+        reblock_nhwc_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, stream>>>(
+            static_cast<const unsigned short*>(z), z2, d.Ci, d.Hp, d.Wp, r.Hp, r.Wp, d.k / r.k, total8);
+        AC_CUDA_TRY(cudaGetLastError());
+        return launch_wgrad_gather_fused(r, z2, dy, dw, workspace, stream);
+    }
     const GatherGeom g = gather_geom(d);
     if (!g.ok) return AC_ERR_UNSUPPORTED;
     char* ws = static_cast<char*>(workspace);

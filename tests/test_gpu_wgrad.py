@@ -551,3 +551,25 @@ def test_sm_budget_layers_side_by_side_match_checker():
         got = w["dw"].double().cpu().numpy().transpose(0, 3, 1, 2)
         assert_dw_close(got, w["want"], "bf16")
         assert_dw_close(got, w["whole"], "bf16")
+
+
+# Few input channels with a pooling block that is a multiple of the stride (k = 4, 8 at stride 2): Z is re-blocked
+# to k' = stride in the workspace (the same inflated map) and the in-kernel gather runs on that.
+FEW_CHANNELS_REBLOCKED = [
+    # N, Ci, Co, H, W, R, S, stride, pad, k
+    (2, 3, 64, 32, 32, 7, 7, 2, 3, 4),
+    (2, 3, 64, 32, 32, 7, 7, 2, 3, 8),
+    (3, 3, 64, 56, 64, 7, 7, 2, 3, 4),
+    (2, 6, 320, 24, 24, 3, 3, 2, 1, 4),
+    (2, 3, 64, 30, 32, 7, 7, 2, 3, 4),       # k does not divide H: the partial last block is re-blocked with the rest
+    (2, 8, 256, 16, 48, 5, 5, 2, 2, 8),
+]
+
+
+@pytest.mark.parametrize("case", FEW_CHANNELS_REBLOCKED)
+def test_few_input_channels_reblocked_match_checker(case):
+    import paper_2409_11902_b200 as ac
+    d = D(*case, "bf16", "nhwc")
+    assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 6
+    err, got, want = wgrad_error_full(d)
+    assert err <= 1e-4 <= TOL_DW["bf16"], err
