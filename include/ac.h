@@ -361,7 +361,12 @@ typedef struct {
                                 tile copies in shared memory at all: the inflated map Xt is written to the
                                 workspace (|X| bytes) and kernel 2 runs on it with k = 1 (described by
                                 the other fields); with a workspace of ac_workspace_bytes_min() bytes
-                                the kernel reads Z itself where it can,
+                                the kernel reads Z itself where it can. For square blocks of 4 and more
+                                the same route is taken with Z re-blocked to a smaller block k' that
+                                divides k, Z'[p][q] = Z[p*k'/k][q*k'/k] (|X| / k'^2 elements; the same
+                                inflated map), where the plan for k' is expected to be faster (fewer
+                                output classes; 64-channel layers pair their taps at k' = 2); `phases`
+                                then counts the classes of that plan,
                                 6: as 5 when taps share columns (both strides multiples of k, k divides H
                                 and W, at most 128 columns, rows of Z a multiple of 16 bytes long): the matrix
                                 is never written to memory; sixteen warps of the kernel build each K-tile

@@ -50,7 +50,8 @@
 namespace ac {
 namespace {
 
-// Xt[n][h][w][c] = Z[n][h / kh][w / kw][c], bf16 NHWC, eight channels (16 bytes) per thread
+// Xt[n][h][w][c] = Z[n][h / kh][w / kw][c] for h < H, w < W, bf16 NHWC, eight channels (16 bytes) per thread.
+// With (H, W) the pooled size of a smaller block k' and kh = kw = k / k' this is Z re-blocked to k'.
 __global__ void __launch_bounds__(256)
 inflate_nhwc_kernel(const uint4* __restrict__ z, uint4* __restrict__ xt, int H, int W, int Hp, int Wp, int C8, int kh,
                     int kw, long long total) {
@@ -447,17 +448,31 @@ bool inflate_problem(const Dims& d, Dims* out) {
     if (d.dtype != AC_BF16 || d.layout != AC_NHWC || (d.kh == 1 && d.kw == 1) || d.max_chain != 0) return false;
     int copies = 0;
     const double direct = tc2_cost_cycles(d, &copies);      // negative: the kernel cannot read this Z at all
-    if (direct >= 0.0 && copies < 2) return false;
-    Dims in = d;
-    in.k = in.kh = in.kw = 1;
-    in.Hp = d.H;
-    in.Wp = d.W;
-    if (in.z_elems() >= (1ll << 40) || (in.z_elems() / 8 + 255) / 256 >= (1ll << 31)) return false;
-    const double inflated = tc2_cost_cycles(in, nullptr);
-    if (inflated < 0.0) return false;
-    const double pass = 6000.0 + 2.0 * (double)(d.z_elems() + in.z_elems()) * 2.9e-4;     // cycles: launch + bytes at ~3.4 KB/clk
-    if (direct >= 0.0 && inflated + pass >= 0.85 * direct) return false;
-    *out = in;
+    // Candidates: the fully inflated map (k' = 1) where the tile needs several copies or cannot be read at all, and,
+    // for square blocks of 4 and more, Z re-blocked to a smaller block k' = k/2, k/4, ... >= 2 (the same inflated
+    // map, see reblocked_dims): sixteen or sixty-four output classes cost more per K-tile than four, and 64-channel
+    // layers pair their taps only when every class agrees on the shifts.
+    double best = -1.0;
+    Dims best_in{};
+    for (int k2 = d.kh == d.kw ? d.k / 2 : 1; k2 >= 1; k2 /= 2) {
+        if (k2 > 1 && (d.k % k2 != 0 || d.k < 4)) continue;
+        if (k2 == 1 && direct >= 0.0 && copies < 2) break;
+        Dims in = d;
+        in.k = in.kh = in.kw = k2;
+        in.Hp = (d.H + k2 - 1) / k2;
+        in.Wp = (d.W + k2 - 1) / k2;
+        if (in.z_elems() >= (1ll << 40) || (in.z_elems() / 8 + 255) / 256 >= (1ll << 31)) continue;
+        int c2 = 0;
+        const double inner = tc2_cost_cycles(in, &c2);
+        if (inner < 0.0) continue;
+        // the pass: a launch, and its bytes at ~3.4 KB per cycle
+        const double cost = inner + 6000.0 + 2.0 * (double)(d.z_elems() + in.z_elems()) * 2.9e-4;
+        if (best < 0.0 || cost < best) { best = cost; best_in = in; }
+        if (k2 == 1) break;
+    }
+    if (best < 0.0) return false;
+    if (direct >= 0.0 && best >= 0.85 * direct) return false;
+    *out = best_in;
     return true;
 }
 
@@ -578,9 +593,10 @@ ac_status launch_wgrad_staged(const Dims& d, const WgradPlan& pl, const void* z,
     ac_status st = AC_OK;
     if (d.dtype == AC_BF16 && d.layout == AC_NHWC) {
         const long long total = in.a.z_elems() / 8;
+        // the inner problem's Z: the inflated map itself (k' = 1) or Z re-blocked to k'
         inflate_nhwc_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
-            static_cast<const uint4*>(z), reinterpret_cast<uint4*>(z_st), d.H, d.W, d.Hp, d.Wp, d.Ci / 8, d.kh, d.kw,
-            total);
+            static_cast<const uint4*>(z), reinterpret_cast<uint4*>(z_st), in.a.Hp, in.a.Wp, d.Hp, d.Wp, d.Ci / 8,
+            d.kh / in.a.kh, d.kw / in.a.kw, total);
         AC_CUDA_TRY(cudaGetLastError());
         return launch_wgrad_tc2(in.a, pl, z_st, dy, dw, workspace, stream);
     }

@@ -257,7 +257,7 @@ def main():
         tfl = d.flops / t_w / 1e6
         gbs = (xb + zb) / t_c / 1e3
         path = {0: "fp32 ALU", 1: "tc", 2: "tc2", 3: "staged", 4: "staged×2", 5: "gather", 6: "gather (in kernel)",
-                7: "tc2 on inflated"}.get(
+                7: "tc2 on re-blocked Z"}.get(
             api.ac_wgrad_plan_info(d)["tensor_core"], "?")
         print(f"| {ci}→{co}, {H}², {R}x{R}/{st} | {cnt} | {path} | {xb / 2**20:.1f} | {zb / 2**20:.1f} | {t_c:.1f} | "
               f"{gbs:.0f} | {gbs / hbm:.2f} | {t_w:.1f} | {tfl:.0f} | {kind} {bound:.0f} | {tfl / bound:.2f} |")

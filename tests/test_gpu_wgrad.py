@@ -573,3 +573,28 @@ def test_few_input_channels_reblocked_match_checker(case):
     assert ac.ac_wgrad_plan_info(d)["tensor_core"] == 6
     err, got, want = wgrad_error_full(d)
     assert err <= 1e-4 <= TOL_DW["bf16"], err
+
+
+# Pooling blocks of 4 and 8: where the cost model prefers it, Z is re-blocked in the workspace to a smaller block
+# k' that divides k (the same inflated map) and the TMA-fed kernel runs with k' (plan code 7, phases = its classes).
+REBLOCKED = [
+    # N, Ci, Co, H, W, R, S, stride, pad, k, classes of the inner plan
+    (16, 64, 64, 56, 56, 3, 3, 1, 1, 4, 4),        # 64 channels: the taps pair up at k' = 2, not at k = 4
+    (16, 64, 64, 56, 56, 3, 3, 1, 1, 8, 4),
+    (32, 256, 256, 14, 14, 3, 3, 1, 1, 4, 4),      # 14 = 3 * 4 + 2: partial blocks at k = 4, none at k' = 2
+    (8, 128, 128, 28, 28, 3, 3, 1, 1, 8, 1),       # all the way to the inflated map
+]
+
+
+@pytest.mark.parametrize("case", REBLOCKED)
+def test_reblocked_pooling_blocks_match_checker(case):
+    import paper_2409_11902_b200 as ac
+    *shape, classes = case
+    d = D(*shape, "bf16", "nhwc")
+    info = ac.ac_wgrad_plan_info(d)
+    assert (info["tensor_core"], info["phases"]) == (7, classes)
+    z, dy = make_wgrad_inputs(d)
+    for nbytes in sorted({ac.ac_workspace_bytes_min(d), ac.ac_workspace_bytes(d)}):
+        got = run_wgrad(d, z, dy, nbytes=nbytes)
+        err = sampled_check(d, got, z, dy, n_samples=512)
+        assert err <= 1e-4, (nbytes, err)
