@@ -121,9 +121,14 @@ def test_plan_info_respects_hardware_limits(ac):
             d = ac.ConvDesc(N, ci, co, H, W, R, S, (st, st), (pd, pd), k, "bf16", "nhwc")
             i = ac.ac_wgrad_plan_info(d)
             assert i["tensor_core"] in (1, 2, 7), d
-            inflated = i["tensor_core"] == 7     # the TMA-fed kernel on an inflated copy of Z kept in the workspace
+            # 7: the TMA-fed kernel on Z re-blocked to a block k2 that divides k (k2 = 1: the inflated map), kept in
+            # the workspace; `phases` counts that plan's classes
+            inflated = i["tensor_core"] == 7
+            k2 = k
             if inflated:
-                assert k > 1 and (H % k or W % k) and pd > 0
+                k2 = st * int(round(i["phases"] ** 0.5)) if i["phases"] > 1 else (1 if st == 1 or k % st else st)
+                assert k > 1 and k % k2 == 0 and k2 < k
+                assert k2 > 1 or ((H % k or W % k) and pd > 0)      # all the way to the inflated map: partial blocks only
             assert 2 <= i["stages"] <= 8
             assert i["smem_bytes"] <= 227 * 1024
             assert i["tmem_columns"] in (32, 64, 128, 256, 512)
@@ -133,7 +138,7 @@ def test_plan_info_respects_hardware_limits(ac):
                 assert i["k_tile"] >= i["band_rows"] * i["row_pitch"]
                 assert i["row_pitch"] >= d.Wo
             else:   # per class: (band_rows / c_h) class rows of row_pitch >= Wo / c_w positions
-                c_h = c_w = 1 if inflated else max(1, k // st)     # a stride above k: one class, phase planes of Z
+                c_h = c_w = max(1, k2 // st)     # a stride above the block: one class, phase planes of Z
                 assert i["phases"] == c_h * c_w <= 64
                 assert i["k_tile"] >= (i["band_rows"] // c_h) * i["row_pitch"]
                 assert i["row_pitch"] >= -(-d.Wo // c_w)
@@ -141,15 +146,20 @@ def test_plan_info_respects_hardware_limits(ac):
             assert i["ctas"] == i["splits"] * i["groups"]
             want = 256 + (i["splits"] * 4 * co * ci * R * S if i["splits"] > 1 else 0)
             if inflated:
-                want = -(-want // 256) * 256 + -(-N * H * W * ci * 2 // 256) * 256
+                want = -(-want // 256) * 256 + -(-N * -(-H // k2) * -(-W // k2) * ci * 2 // 256) * 256
                 assert ac.ac_workspace_bytes_min(d) <= want
             assert ac.ac_workspace_bytes(d) == want
     # 64 input channels, 3x3, k = 2: the nine taps pair up into five accumulator tiles in one CTA
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 64, 64, 56, 56, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
     assert (i["tensor_core"], i["units_per_cta"], i["groups"]) == (2, 5, 1)
-    # k = 8 at stride 1: 64 output classes, still the TMA-fed kernel
-    i = ac.ac_wgrad_plan_info(ac.ConvDesc(256, 128, 128, 64, 64, 3, 3, (1, 1), (1, 1), 8, "bf16", "nhwc"))
-    assert (i["tensor_core"], i["phases"]) == (2, 64)
+    # k = 8 at stride 1: 64 output classes on the TMA-fed kernel when the workspace has no room for a re-blocked Z,
+    # four classes on Z re-blocked to 2 x 2 when it has (k = 4: sixteen classes, read directly)
+    d8 = ac.ConvDesc(256, 128, 128, 64, 64, 3, 3, (1, 1), (1, 1), 8, "bf16", "nhwc")
+    i = ac.ac_wgrad_plan_info(d8)
+    assert (i["tensor_core"], i["phases"]) == (7, 4)
+    assert ac.ac_workspace_bytes(d8) - ac.ac_workspace_bytes_min(d8) >= 256 * 32 * 32 * 128 * 2 - 64 * 4 * 128 * 128 * 9
+    i = ac.ac_wgrad_plan_info(ac.ConvDesc(256, 128, 128, 64, 64, 3, 3, (1, 1), (1, 1), 4, "bf16", "nhwc"))
+    assert (i["tensor_core"], i["phases"]) == (2, 16)
     # a small map that k does not divide, with padding (partial pooling blocks that taps read past): the
     # TMA-fed kernel runs on the inflated map; without padding, or on a larger map, it reads Z itself
     i = ac.ac_wgrad_plan_info(ac.ConvDesc(64, 512, 512, 7, 7, 3, 3, (1, 1), (1, 1), 2, "bf16", "nhwc"))
